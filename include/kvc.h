@@ -1,0 +1,180 @@
+/*
+ * kvc -- the KVCompose compression pass over a prefilled KV cache, for NVIDIA B200 (sm_100a).
+ *
+ * Given, for every layer, the cached keys/values K, V in R^{Hkv x N x d} (Sec. 3.1 of the paper)
+ * and the post-RoPE queries of a scoring window (the "task tokens" of Sec. 3.2.2), the pass
+ *   (1) scores every cached token per layer and KV head          -- kvc_score    (Eqs. 3, 14-16)
+ *   (2) sorts the tokens of every head by score, aligns the rank-k token of each head into the
+ *       k-th composite token and gives it a composite score      -- kvc_compose  (Eqs. 17-19)
+ *   (3) splits one global budget of token slots over the layers  -- kvc_allocate (Eqs. 20-22)
+ *   (4) copies the retained K/V rows into a dense cache that is uniform across the heads of a
+ *       layer                                                    -- kvc_gather   (Eqs. 23-24)
+ * kvc_compress runs (1)-(4) back to back on one stream without a host synchronisation.
+ *
+ * General conventions
+ *   - Plain C ABI.  Every data pointer is a DEVICE pointer owned by the caller unless it is
+ *     marked "host".  The library allocates no device memory and frees none: scratch space comes
+ *     from the caller's workspace (kvc_workspace_size bytes, 256-byte aligned).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the default stream);
+ *     calls return without synchronising.  The return value reports errors the host can see
+ *     (bad arguments, a failed launch); kvc_last_error() then holds a message.
+ *   - Inputs are never modified.  Indices are 0-based.  Sequences of a batch are independent:
+ *     each has its own pool and its own budget (the paper has no batch dimension).
+ *   - Finite inputs are a precondition; NaN/Inf in Q or K give unspecified scores.
+ *   - All entry points need a CUDA device of compute capability 10.0; there is no CPU path.
+ */
+#ifndef KVC_H_
+#define KVC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define KVC_API __attribute__((visibility("default")))
+#else
+#define KVC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KVC_OK = 0,
+  KVC_ERR_INVALID_ARG = -1, /* NULL pointer, inconsistent sizes, misaligned buffer, bad budget */
+  KVC_ERR_UNSUPPORTED = -2, /* shape outside what the kernels handle (see kvc_desc) */
+  KVC_ERR_WORKSPACE = -3,   /* workspace missing, misaligned or smaller than kvc_workspace_size */
+  KVC_ERR_CUDA = -4,        /* a CUDA runtime call failed; message in kvc_last_error() */
+  KVC_ERR_TIMEOUT = -5      /* device_status only: a bounded device-side wait gave up */
+} kvc_status;
+
+typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
+
+/* Aggregation operator of Eqs. 14, 15, 19: max-pooling or average-pooling. */
+typedef enum { KVC_AGG_MAX = 0, KVC_AGG_MEAN = 1 } kvc_agg;
+
+#define KVC_MAX_LAYERS 128
+
+/*
+ * Problem description (Sec. 3.1: L layers, K, V in R^{Hkv x N x d}; Sec. 2.2: G = Hq / Hkv).
+ *
+ * Layouts, per layer l (one device pointer per layer):
+ *   Q^(l)  [batch, n_q_heads,  window, head_dim]   element strides q_stride  = (batch, head, row)
+ *   K^(l), V^(l) [batch, n_kv_heads, n_ctx, head_dim]  element strides kv_stride = (batch, head, token)
+ * The last dimension is contiguous; every row must start on a 16-byte boundary.  A stride of 0
+ * in slot 0 of either array means "dense" and all three are filled in from the shape.
+ */
+typedef struct {
+  int32_t n_layers;   /* L, 1..KVC_MAX_LAYERS; L * batch <= 65535 */
+  int32_t batch;      /* independent sequences, >= 1 */
+  int32_t n_q_heads;  /* Hq */
+  int32_t n_kv_heads; /* Hkv */
+  int32_t head_dim;   /* d: 64 or 128 */
+  int32_t window;     /* w = M: scoring-query rows per query head (Sec. 3.2.2), >= 1 */
+  int64_t n_ctx;      /* N cached tokens per sequence, 1 <= N < 2^31 */
+  int64_t q_pos0;     /* absolute position of window row 0.  Row m attends to key c iff
+                         c <= q_pos0 + m (the model's causal mask).  N - w scores the last w
+                         context tokens against the context; any value >= N disables masking
+                         (task tokens that follow the context).  Must be >= 0. */
+  int32_t dtype;      /* kvc_dtype of Q, K, V and of the compressed K', V' */
+  float scale;        /* logit scale; <= 0 selects 1/sqrt(head_dim) (Eq. 3) */
+  int32_t agg_task;   /* Eq. 14, over the window rows.   Paper default: KVC_AGG_MAX  */
+  int32_t agg_group;  /* Eq. 15, over the G query heads. Paper default: KVC_AGG_MEAN */
+  int32_t agg_head;   /* Eq. 19, over the KV heads.      Paper default: KVC_AGG_MEAN */
+  int32_t augment_head_mean; /* Eq. 16: add the mean over KV heads to every head's score (default 1) */
+  const int32_t* q_to_kv;    /* HOST pointer, n_q_heads entries: KV head of each query head;
+                                NULL = j / G with G = Hq / Hkv (Sec. 3.2.2, the reshape before
+                                Eq. 15; then Hq % Hkv must be 0).  Every KV head needs >= 1 member. */
+  int64_t q_stride[3];
+  int64_t kv_stride[3];
+} kvc_desc;
+
+/* Fill *desc with the paper's defaults for the given shape (dense strides, q_pos0 = N - w,
+ * scale 1/sqrt(d), max / mean / mean, head-mean on, contiguous GQA groups). */
+KVC_API void kvc_desc_init(kvc_desc* desc, int32_t n_layers, int32_t batch, int32_t n_q_heads,
+                   int32_t n_kv_heads, int32_t head_dim, int64_t n_ctx, int32_t window,
+                   int32_t dtype);
+
+/* B_total = floor((1 - r_target) * L * N), per sequence (Eq. 21).  The product is evaluated in
+ * double and nudged up by a relative 1e-12 before the floor so that decimal ratios such as 0.8
+ * behave as in exact arithmetic.  Returns -1 on a bad descriptor or r_target outside [0, 1]. */
+KVC_API int64_t kvc_budget_from_ratio(const kvc_desc* desc, double r_target);
+
+/* Bytes of scratch any entry point below may need for this problem and budget (host call). */
+KVC_API kvc_status kvc_workspace_size(const kvc_desc* desc, int64_t budget, size_t* bytes);
+
+/*
+ * Token importance (Sec. 3.2.2).  For layer l, sequence b, query head j, window row m:
+ *   A[m, c] = softmax over the visible keys c of  scale * <q[j, m], k[kv(j), c]>      (Eq. 3)
+ *   S_task[j, c]  = agg_task over m of A[m, c]   (a masked entry counts as 0)          (Eq. 14)
+ *   S_group[h, c] = agg_group over the query heads of KV head h                        (Eq. 15)
+ *   S[h, c] = S_group[h, c] + mean over the KV heads i of S_group[i, c]                (Eq. 16)
+ * q, k: HOST arrays of n_layers device pointers.  scores: [L, batch, Hkv, N] fp32, dense.
+ * bf16 inputs are multiplied exactly and accumulated in fp32; the attention tensor A is
+ * never written to memory.
+ */
+KVC_API kvc_status kvc_score(const kvc_desc* desc, const void* const* q, const void* const* k,
+                     float* scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Ranking and composite tokens (Sec. 3.3).  For every (l, b, h):
+ *   idx[l, b, h, :] = positions 0..N-1 sorted by score, descending; equal scores keep the
+ *                     smaller position first                                            (Eq. 17)
+ *   composite token k of layer l = { idx[l, b, h, k] : h }  (column k of idx, no copy)
+ *   composite[l, b, k] = agg_head over h of scores[l, b, h, idx[l, b, h, k]]       (Eqs. 18-19)
+ * The mean is evaluated in fp32 as ((S'_0 + S'_1) + ...) / Hkv, heads in ascending order.
+ * idx: [L, batch, Hkv, N] int32.  composite: [L, batch, N] fp32, non-increasing in k.
+ * Scores must be non-negative and finite (what kvc_score produces).
+ */
+KVC_API kvc_status kvc_compose(const kvc_desc* desc, const float* scores, int32_t* idx, float* composite,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Layer-adaptive budget (Sec. 3.3, Eqs. 20-22).  Per sequence b, all composite[l, b, k] form one
+ * pool; the `budget` largest are kept, ties resolved by the total order (score descending,
+ * layer ascending, k ascending); n_keep[b, l] = how many of them lie in layer l.
+ *   n_keep:  [batch, L] int32,  sum over l == budget exactly, 0 <= n_keep <= N
+ *   offsets: [batch, L + 1] int64, exclusive prefix sum of n_keep (offsets[b, L] == budget)
+ * composite must be non-increasing in k within a layer (what kvc_compose produces) and
+ * non-negative.  0 <= budget <= L * N.
+ */
+KVC_API kvc_status kvc_allocate(const kvc_desc* desc, const float* composite, int64_t budget,
+                        int32_t* n_keep, int64_t* offsets, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/*
+ * Compaction (Eqs. 23-24): K'[l][h, k, :] = K[l][h, idx[l, h, k], :] for k < n_keep[l]; V alike.
+ * k_out, v_out: [batch, budget * Hkv * d] elements of the cache dtype.  Within sequence b, layer l
+ * starts at element offsets[b, l] * Hkv * d and is a dense [Hkv, n_keep[b, l], d] tensor, rows in
+ * descending score order.  Rows are copied bit for bit.  n_keep / offsets are read on the device
+ * (no host synchronisation); the output size is known beforehand because sum_l n_keep == budget.
+ */
+KVC_API kvc_status kvc_gather(const kvc_desc* desc, const void* const* k, const void* const* v,
+                      const int32_t* idx, const int32_t* n_keep, const int64_t* offsets,
+                      int64_t budget, void* k_out, void* v_out, void* stream);
+
+/*
+ * The whole pass, stream-ordered.  idx_out [L, batch, Hkv, N], scores_out [L, batch, Hkv, N] and
+ * composite_out [L, batch, N] may be NULL (the workspace then holds them).  device_status, if
+ * not NULL, receives KVC_OK or a negative kvc_status detected on the device.
+ */
+KVC_API kvc_status kvc_compress(const kvc_desc* desc, const void* const* q, const void* const* k,
+                        const void* const* v, int64_t budget, void* k_out, void* v_out,
+                        int32_t* n_keep, int64_t* offsets, int32_t* idx_out, float* scores_out,
+                        float* composite_out, int32_t* device_status, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/* Message of the last error returned on this thread (static storage; never NULL). */
+KVC_API const char* kvc_last_error(void);
+
+/* Number of kernels the library has launched on this thread since the last call with reset != 0
+ * (a host-side counter for benchmarks; it does not touch the device). */
+KVC_API int64_t kvc_launch_count(int32_t reset);
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+KVC_API int32_t kvc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVC_H_ */

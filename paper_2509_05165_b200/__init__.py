@@ -1,0 +1,28 @@
+"""KVCompose compression pass for NVIDIA B200: thin Python binding over the C-ABI library.
+
+Every step runs in the CUDA kernels of ``libkvc.so``; this package only marshals
+arguments (torch tensors are used for device memory and streams).
+"""
+from .binding import (  # noqa: F401
+    AGG_MAX,
+    AGG_MEAN,
+    BF16,
+    F32,
+    KvcDesc,
+    KvcError,
+    desc_from_config,
+    kvc_allocate,
+    kvc_budget_from_ratio,
+    kvc_compose,
+    kvc_compress,
+    kvc_desc_init,
+    kvc_gather,
+    kvc_last_error,
+    kvc_launch_count,
+    kvc_score,
+    kvc_version,
+    kvc_workspace_size,
+    library_path,
+    CompressOutputs,
+    compress,
+)

@@ -1,0 +1,107 @@
+// Internal declarations shared by the kvc translation units (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvc.h"
+
+namespace kvc {
+
+constexpr int kMaxQHeads = 256;
+constexpr int kMaxKvHeads = 128;
+
+// Resolved problem: the public descriptor with defaults filled in and the GQA map expanded.
+struct Problem {
+  int L, Bt, Hq, Hkv, d, w;
+  long long N, q_pos0;
+  int dtype;  // kvc_dtype
+  float scale;
+  int agg_task, agg_group, agg_head, augment;
+  long long qs[3], kvs[3];        // element strides (batch, head, row/token)
+  int elem_bytes;                 // 2 or 4
+  int max_group;                  // largest number of query heads sharing one KV head
+  bool contiguous_groups;         // q_to_kv[j] == j / G
+};
+
+// Query heads grouped by KV head: members of KV head h are qh[begin[h] .. begin[h+1]).
+struct GroupMap {
+  int16_t begin[kMaxKvHeads + 1];
+  int16_t qh[kMaxQHeads];
+};
+
+// Per-layer device pointers, passed by value to kernels.
+struct LayerPtrs {
+  const void* p[KVC_MAX_LAYERS];
+};
+
+void set_error(const char* fmt, ...);
+kvc_status check_cuda(cudaError_t e, const char* what);
+void count_launch(int n = 1);
+
+#define KVC_CUDA(call)                                        \
+  do {                                                        \
+    kvc_status _s = ::kvc::check_cuda((call), #call);         \
+    if (_s != KVC_OK) return _s;                              \
+  } while (0)
+
+#define KVC_LAUNCH_CHECK(name)                                \
+  do {                                                        \
+    ::kvc::count_launch();                                    \
+    kvc_status _s = ::kvc::check_cuda(cudaGetLastError(), name); \
+    if (_s != KVC_OK) return _s;                              \
+  } while (0)
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// ---- score ------------------------------------------------------------------------------------
+// Scratch bytes the scoring step needs.
+size_t score_workspace_bytes(const Problem& P);
+// Eqs. 3, 14-16: writes scores [L, Bt, Hkv, N].
+kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
+                        float* scores, void* ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- rank + compose ---------------------------------------------------------------------------
+size_t compose_workspace_bytes(const Problem& P);
+// Eqs. 17-19: idx [L, Bt, Hkv, N], composite [L, Bt, N].
+kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, float* composite,
+                          void* ws, size_t ws_bytes, cudaStream_t st);
+
+// ---- allocate ---------------------------------------------------------------------------------
+size_t allocate_workspace_bytes(const Problem& P);
+// Eqs. 20-22: n_keep [Bt, L], offsets [Bt, L + 1].
+kvc_status launch_allocate(const Problem& P, const float* composite, long long budget,
+                           int32_t* n_keep, long long* offsets, void* ws, size_t ws_bytes,
+                           cudaStream_t st);
+
+// ---- gather -----------------------------------------------------------------------------------
+// Eqs. 23-24.
+kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& v, const int32_t* idx,
+                         const int32_t* n_keep, const long long* offsets, long long budget,
+                         void* k_out, void* v_out, cudaStream_t st);
+
+// Order-preserving map from an fp32 score to an unsigned key whose ASCENDING order is the
+// score's DESCENDING order; -0 is folded onto +0 so that equal scores get equal keys.
+__host__ __device__ inline uint32_t score_to_key(float s) {
+#ifdef __CUDA_ARCH__
+  uint32_t b = __float_as_uint(s);
+#else
+  union { float f; uint32_t u; } cv; cv.f = s; uint32_t b = cv.u;
+#endif
+  if (b == 0x80000000u) b = 0u;
+  uint32_t asc = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  return ~asc;
+}
+
+__host__ __device__ inline float key_to_score(uint32_t key) {
+  uint32_t asc = ~key;
+  uint32_t b = (asc & 0x80000000u) ? (asc & 0x7fffffffu) : ~asc;
+#ifdef __CUDA_ARCH__
+  return __uint_as_float(b);
+#else
+  union { float f; uint32_t u; } cv; cv.u = b; return cv.f;
+#endif
+}
+
+}  // namespace kvc

@@ -1,0 +1,248 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded
+inputs -- element by element at sizes the oracle finishes in seconds, covering several tiles,
+ragged tails, both dtypes, both head sizes, every aggregator, custom GQA maps, strides, batches
+and the degenerate budgets."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import paper_2509_05165_b200 as kvc
+from paper_2509_05165_b200 import workloads as W
+from paper_2509_05165_b200.binding import alloc_outputs
+
+import parity as Pz
+
+
+def _cuda():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return torch.device("cuda:0")
+
+
+def _host(t):
+    return t.detach().cpu().numpy()
+
+
+def run_staged(wl, desc, budget):
+    """The four stage entry points one after another; returns host copies of every output."""
+    dev = wl.k[0].device
+    out = alloc_outputs(desc, budget, wl.k[0].dtype, dev)
+    kvc.kvc_score(desc, wl.q, wl.k, out.scores, out.workspace)
+    kvc.kvc_compose(desc, out.scores, out.idx, out.composite, out.workspace)
+    kvc.kvc_allocate(desc, out.composite, budget, out.n_keep, out.offsets, out.workspace)
+    kvc.kvc_gather(desc, wl.k, wl.v, out.idx, out.n_keep, out.offsets, budget, out.k_out, out.v_out)
+    torch.cuda.synchronize()
+    return out
+
+
+def run_fused(wl, desc, budget, keep=True):
+    out = kvc.compress(wl.q, wl.k, wl.v, desc, budget, keep_intermediates=keep)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    return out
+
+
+def check_all(wl, desc, budget, e2e_strict=False, check_e2e=True):
+    st = run_staged(wl, desc, budget)
+    fu = run_fused(wl, desc, budget)
+    # the fused entry runs the same kernels: identical bits
+    for name in ("scores", "idx", "composite", "n_keep", "offsets", "k_out", "v_out"):
+        a, b = getattr(st, name), getattr(fu, name)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), "fused != staged for " + name
+    S = _host(fu.scores); idx = _host(fu.idx); I = _host(fu.composite)
+    n_keep = _host(fu.n_keep); off = _host(fu.offsets)
+    # P1: scores against the all-double oracle
+    S_def = Pz.oracle_scores(wl, desc)
+    worst = Pz.assert_scores_close(S, S_def)
+    # P2: staged, exact
+    Pz.assert_rank_exact(S, idx)
+    Pz.assert_compose_exact(S, idx, I, desc.agg_head)
+    Pz.assert_allocate_exact(I, budget, n_keep, off)
+    Pz.assert_gather_exact(wl, desc, idx, n_keep, off, fu.k_out, fu.v_out)
+    # invariants
+    assert np.all(np.sort(idx, axis=-1) == np.arange(desc.n_ctx)[None, None, None, :])
+    assert np.all(np.diff(I, axis=-1) <= 0)
+    # P3: end to end against the all-double oracle, tolerance-aware
+    rep = None
+    if check_e2e:
+        rep = Pz.end_to_end_report(S_def, idx)
+        assert rep["order_violations"] == 0, rep
+        assert rep["max_gap_at_diff"] < 2 * Pz.SCORE_RTOL, rep
+        if e2e_strict:
+            assert rep["n_diff"] == 0, rep
+    # a fused call that keeps no intermediates gives the same compressed cache
+    lean = run_fused(wl, desc, budget, keep=False)
+    assert torch.equal(lean.k_out.view(torch.uint8), fu.k_out.view(torch.uint8))
+    assert torch.equal(lean.n_keep, fu.n_keep)
+    return worst, rep
+
+
+def test_tiny_config_fp32():
+    """The tiny fp32 configuration, whole pass, every element."""
+    dev = _cuda()
+    cfg = W.TINY
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    assert cfg.budget == 256
+    check_all(wl, desc, cfg.budget)
+
+
+def test_tiny_config_separated_scores_strict_order():
+    """Unit-variance inputs give well separated scores: the GPU order must equal the oracle's."""
+    dev = _cuda()
+    cfg = W.TINY.replace(elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    _, rep = check_all(wl, desc, cfg.budget)
+    assert rep["n_diff"] <= 2, rep     # an exact tie in double is the only admissible difference
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
+def test_ragged_multi_tile(dtype, d):
+    """N spans several tiles with a ragged tail; GQA group 4; window 32; causal window mask."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("ragged", 3, 8, 2, d, 1500, 32, dtype=dtype, retention=0.3, elem_std=1.0,
+                           hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    check_all(wl, desc, cfg.budget)
+
+
+@pytest.mark.parametrize("agg_task,agg_group,agg_head,augment",
+                         [(0, 0, 0, 0), (1, 1, 1, 1), (0, 1, 1, 0), (1, 0, 0, 1), (0, 0, 1, 1)])
+def test_aggregator_variants(agg_task, agg_group, agg_head, augment):
+    dev = _cuda()
+    cfg = W.WorkloadConfig("agg", 2, 6, 2, 64, 700, 8, dtype="bf16", retention=0.5, elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg, agg_task=agg_task, agg_group=agg_group, agg_head=agg_head,
+                                augment_head_mean=augment)
+    check_all(wl, desc, cfg.budget)
+
+
+@pytest.mark.parametrize("q_pos0_kind", ["none", "middle", "zero"])
+def test_mask_positions(q_pos0_kind):
+    """No mask (task tokens after the context), a window in the middle, and a window at 0."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("mask", 2, 4, 2, 64, 333, 16, dtype="f32", retention=0.4, elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    q_pos0 = {"none": cfg.n_ctx + 5, "middle": 100, "zero": 0}[q_pos0_kind]
+    desc = kvc.desc_from_config(cfg, q_pos0=q_pos0)
+    check_all(wl, desc, cfg.budget)
+
+
+def test_explicit_group_map_and_scale():
+    dev = _cuda()
+    cfg = W.WorkloadConfig("map", 2, 6, 3, 64, 400, 8, dtype="bf16", retention=0.25, elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    m = (ctypes.c_int32 * 6)(2, 0, 1, 1, 0, 2)
+    desc = kvc.desc_from_config(cfg, scale=0.2)
+    desc.q_to_kv = ctypes.cast(m, ctypes.POINTER(ctypes.c_int32))
+    check_all(wl, desc, cfg.budget)
+    # uneven groups: KV head 0 has 4 query heads, head 1 and 2 have one each
+    m2 = (ctypes.c_int32 * 6)(0, 0, 1, 0, 2, 0)
+    desc.q_to_kv = ctypes.cast(m2, ctypes.POINTER(ctypes.c_int32))
+    check_all(wl, desc, cfg.budget)
+
+
+def test_batch_and_strided_inputs():
+    """Two sequences; K/V/Q are views into larger buffers (non-dense batch/head/token strides)."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("strided", 2, 4, 2, 64, 300, 8, batch=2, dtype="bf16", retention=0.35, elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    Bt, Hkv, N, d, Hq, w = 2, 2, 300, 64, 4, 8
+    k2, v2, q2 = [], [], []
+    for l in range(cfg.n_layers):
+        kb = torch.zeros((Bt, Hkv + 1, N + 7, 2 * d), dtype=wl.k[l].dtype, device=dev)
+        vb = torch.zeros_like(kb)
+        qb = torch.zeros((Bt, Hq, w + 3, d + 8), dtype=wl.q[l].dtype, device=dev)
+        kb[:, :Hkv, :N, :d] = wl.k[l]; vb[:, :Hkv, :N, :d] = wl.v[l]; qb[:, :, :w, :d] = wl.q[l]
+        k2.append(kb[:, :Hkv, :N, :d]); v2.append(vb[:, :Hkv, :N, :d]); q2.append(qb[:, :, :w, :d])
+    desc = kvc.desc_from_config(cfg)
+    for i in range(3):
+        desc.kv_stride[i] = k2[0].stride(i)
+        desc.q_stride[i] = q2[0].stride(i)
+    dense = run_fused(wl, kvc.desc_from_config(cfg), cfg.budget)
+    strided = run_fused(W.Workload(cfg, q2, k2, v2), desc, cfg.budget)
+    for name in ("scores", "idx", "composite", "n_keep", "offsets", "k_out", "v_out"):
+        assert torch.equal(getattr(dense, name).view(torch.uint8), getattr(strided, name).view(torch.uint8)), name
+    check_all(wl, kvc.desc_from_config(cfg), cfg.budget)
+
+
+@pytest.mark.parametrize("N,w", [(1, 1), (5, 8), (127, 4), (128, 4), (129, 4), (1024, 16), (1025, 16)])
+def test_small_and_boundary_lengths(N, w):
+    dev = _cuda()
+    cfg = W.WorkloadConfig("edge", 2, 2, 1, 64, N, w, dtype="f32", retention=0.5, elem_std=1.0,
+                           n_sinks=min(4, N), hh_frac=0.0 if N < 200 else 0.01)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    assert desc.q_pos0 == max(N - w, 0)
+    check_all(wl, desc, cfg.budget)
+
+
+def test_degenerate_budgets():
+    dev = _cuda()
+    cfg = W.WorkloadConfig("budget", 3, 4, 2, 64, 200, 8, dtype="bf16", elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    total = cfg.n_layers * cfg.n_ctx
+    for budget in (0, 1, total - 1, total):
+        st = run_fused(wl, desc, budget)
+        n_keep = _host(st.n_keep)
+        assert n_keep.sum() == budget
+        Pz.assert_allocate_exact(_host(st.composite), budget, n_keep, _host(st.offsets))
+        Pz.assert_gather_exact(wl, desc, _host(st.idx), n_keep, _host(st.offsets), st.k_out, st.v_out)
+    # nothing evicted: every head's compressed K is a permutation of its rows
+    st = run_fused(wl, desc, total)
+    for l in range(cfg.n_layers):
+        got = st.k_out[0].view(cfg.n_layers, 2, cfg.n_ctx, 64)[l]
+        for h in range(2):
+            a = sorted(map(bytes, Pz.raw_numpy(got[h])))
+            b = sorted(map(bytes, Pz.raw_numpy(wl.k[l][0, h])))
+            assert a == b
+
+
+def test_exact_ties_are_broken_by_position_and_layer():
+    """All keys identical except a sparse perturbed set: long runs of exactly equal scores.  The
+    order must put equal scores in increasing position, and the budget must be handed out in
+    layer order among equal composite scores."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("ties", 4, 8, 2, 64, 900, 8, dtype="bf16", retention=0.3, hh_mode="ties",
+                           hh_frac=0.01, elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    fu = run_fused(wl, desc, cfg.budget)
+    S = _host(fu.scores); idx = _host(fu.idx)
+    n_equal = int((np.diff(np.take_along_axis(S, idx.astype(np.int64), axis=-1), axis=-1) == 0).sum())
+    assert n_equal > S.size // 2, "the tie workload should produce long runs of equal scores"
+    check_all(wl, desc, cfg.budget, check_e2e=False)
+    # planted composite ties across layers: allocation follows (score desc, layer asc, k asc)
+    I = torch.ones((4, 1, 900), device=dev)
+    I[2, 0, :10] = 2.0
+    n_keep = torch.empty((1, 4), dtype=torch.int32, device=dev)
+    off = torch.empty((1, 5), dtype=torch.int64, device=dev)
+    ws = torch.empty(kvc.kvc_workspace_size(desc, 1000), dtype=torch.uint8, device=dev)
+    kvc.kvc_allocate(desc, I, 1000, n_keep, off, ws)
+    assert n_keep.cpu().tolist() == [[900, 90, 10, 0]]
+    assert off.cpu().tolist() == [[0, 900, 990, 1000, 1000]]
+
+
+def test_argument_errors_are_reported_not_launched():
+    dev = _cuda()
+    cfg = W.WorkloadConfig("err", 1, 2, 1, 64, 64, 4, dtype="f32", elem_std=1.0)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    out = alloc_outputs(desc, 10, torch.float32, dev)
+    small = torch.empty(256, dtype=torch.uint8, device=dev)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_compress(desc, wl.q, wl.k, wl.v, 10, out.k_out, out.v_out, out.n_keep, out.offsets,
+                         workspace=small)
+    assert e.value.status == -3
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_compress(desc, wl.q, wl.k, wl.v, 65, out.k_out, out.v_out, out.n_keep, out.offsets,
+                         workspace=out.workspace)
+    assert e.value.status == -1
+    torch.cuda.synchronize()
