@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the KVCompose compression pass on B200.
+
+One "step" is one whole pass (score -> rank/compose -> allocate -> gather, the fused
+kvc_compress entry) over one synthetic prefilled KV cache.  The default workload is the
+LLaMA-3.1-8B-shaped cache at N = 32768, window 32, 25 % retention (the configuration the
+>= 70 %-of-HBM-roofline target is stated on); --workload picks another one.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--retention R]
+  python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...   (N > 1)
+  python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
+
+Prints ONE JSON line on rank 0.  Multi-GPU: every rank compresses its own sequence (weak
+scaling, no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "context_tokens_per_sec_compressed_end_to_end"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="kvc", choices=["kvc", "reference"])
+    ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--retention", type=float, default=None)
+    ap.add_argument("--n-ctx", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--elem-std", type=float, default=None)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU work of the oracle leg")
+    return ap.parse_args()
+
+
+def pick_config(args):
+    from paper_2509_05165_b200 import workloads as W
+
+    cfg = W.CONFIGS[args.workload]
+    kw = {}
+    if args.retention is not None:
+        kw["retention"] = args.retention
+    if args.n_ctx is not None:
+        kw["n_ctx"] = args.n_ctx
+    if args.batch is not None:
+        kw["batch"] = args.batch
+    if args.elem_std is not None:
+        kw["elem_std"] = args.elem_std
+    return cfg.replace(**kw) if kw else cfg
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:  # noqa: BLE001
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(cfg):
+    """Bytes the method has to move per pass (all sequences of this rank)."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    kv = cfg.n_layers * cfg.n_kv_heads * cfg.n_ctx * cfg.head_dim * e
+    q = cfg.n_layers * cfg.n_q_heads * cfg.window * cfg.head_dim * e
+    rho = cfg.budget / float(cfg.n_layers * cfg.n_ctx)
+    return dict(score=cfg.batch * (kv + q), gather=cfg.batch * 4 * rho * kv,
+                total=cfg.batch * (kv * (1 + 4 * rho) + q))
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "200"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:  # noqa: BLE001
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        time.sleep(0.25)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:  # noqa: BLE001
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def gpu_id(local_rank):
+    """nvidia-smi identifier of the torch device (the UUID survives CUDA_VISIBLE_DEVICES remapping)."""
+    try:
+        return "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:  # noqa: BLE001
+        return str(local_rank)
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(cfg, n_layers_sample):
+    """Host copies of the first layers of the workload, in the form the oracle takes."""
+    from paper_2509_05165_b200 import workloads as W
+
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    wl = W.make_workload(cfg.replace(batch=1), dev, layers=range(n_layers_sample))
+    q = np.stack([t[0].float().cpu().numpy() for t in wl.q])
+    k = np.stack([t[0].float().cpu().numpy() for t in wl.k])
+    view = torch.int16 if cfg.dtype == "bf16" else torch.float32
+    kr = np.stack([t[0].view(view).cpu().numpy() for t in wl.k])
+    vr = np.stack([t[0].view(view).cpu().numpy() for t in wl.v])
+    return q, k, kr, vr
+
+
+def time_oracle(cfg, q, k, kr, vr):
+    import oracle
+
+    Ls = q.shape[0]
+    budget = int(cfg.retention * Ls * cfg.n_ctx)
+    t0 = time.perf_counter()
+    oracle.compress(q, k, kr, vr, 1.0 / np.sqrt(cfg.head_dim), cfg.n_ctx - cfg.window, budget,
+                    want_scores=False)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, target_seconds):
+    """The oracle as it stands, on the host cores, on the first layers of the same workload."""
+    import oracle
+
+    cores = host_cores()
+    oracle.set_threads(cores)
+    q, k, kr, vr = oracle_sample(cfg, 1)
+    t1 = time_oracle(cfg, q, k, kr, vr)
+    Ls = int(max(1, min(cfg.n_layers, round(target_seconds / max(t1, 1e-3)))))
+    if Ls > 1:
+        q, k, kr, vr = oracle_sample(cfg, Ls)
+        t = time_oracle(cfg, q, k, kr, vr)
+    else:
+        t = t1
+    per_pass = t * cfg.n_layers / Ls          # linear in the number of layers
+    return dict(value=cfg.n_ctx / per_pass, unit=UNIT, cores=cores, kind="oracle",
+                sample="%d of %d layers of %s, one sequence, whole pass incl. gather: %.2f s measured, "
+                       "scaled linearly to all layers" % (Ls, cfg.n_layers, cfg.name, t),
+                seconds_measured=t)
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+
+    cfg = pick_config(args)
+    cores = host_cores()
+    oracle.set_threads(cores)
+    Ls = min(cfg.n_layers, 2)
+    q, k, kr, vr = oracle_sample(cfg, Ls)
+    for _ in range(args.warmup):
+        time_oracle(cfg, q, k, kr, vr)
+    times = [time_oracle(cfg, q, k, kr, vr) for _ in range(args.steps)]
+    t_step = sum(times) / len(times)
+    value = cfg.n_ctx / (t_step * cfg.n_layers / Ls)
+    sample = "%d of %d layers of %s per step, one sequence, scaled linearly to all layers" % (Ls, cfg.n_layers, cfg.name)
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=t_step * 1e3 * cfg.n_layers / Ls, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=workload_config(cfg, 1),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def workload_config(cfg, world):
+    return dict(workload=cfg.name, n_layers=cfg.n_layers, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                head_dim=cfg.head_dim, n_ctx=cfg.n_ctx, window=cfg.window, batch_per_gpu=cfg.batch,
+                retention=cfg.retention, budget_per_sequence=cfg.budget, elem_std=cfg.elem_std,
+                sequences_total=cfg.batch * world,
+                l2="inputs (%.2f GB of K/V per GPU) exceed the 126 MB L2; no flush needed" %
+                   (2 * cfg.batch * cfg.n_layers * cfg.n_kv_heads * cfg.n_ctx * cfg.head_dim *
+                    (2 if cfg.dtype == "bf16" else 4) / 1e9))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import paper_2509_05165_b200 as kvc
+    from paper_2509_05165_b200 import workloads as W
+    from paper_2509_05165_b200.binding import alloc_outputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = pick_config(args).replace(seed=rank)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg)
+    budget = cfg.budget
+    out = alloc_outputs(desc, budget, wl.k[0].dtype, dev, keep_intermediates=False)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        kvc.kvc_compress(desc, wl.q, wl.k, wl.v, budget, out.k_out, out.v_out, out.n_keep, out.offsets,
+                         None, None, None, out.device_status, out.workspace, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(gpu_id(local_rank)) if rank == 0 else None
+    kvc.kvc_launch_count(reset=True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    barrier()
+    launches = kvc.kvc_launch_count()
+    ms_total = ev0.elapsed_time(ev1)
+    assert int(out.device_status.item()) == 0
+
+    # ---- per-stage timing (the stage entry points, events between them)
+    inter = alloc_outputs(desc, budget, wl.k[0].dtype, dev, keep_intermediates=True, workspace=out.workspace)
+    names = ["score", "compose", "allocate", "gather"]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    barrier()
+    for s in range(args.steps):
+        e = evs[s]
+        e[0].record(stream)
+        kvc.kvc_score(desc, wl.q, wl.k, inter.scores, out.workspace, stream); e[1].record(stream)
+        kvc.kvc_compose(desc, inter.scores, inter.idx, inter.composite, out.workspace, stream); e[2].record(stream)
+        kvc.kvc_allocate(desc, inter.composite, budget, inter.n_keep, inter.offsets, out.workspace, stream); e[3].record(stream)
+        kvc.kvc_gather(desc, wl.k, wl.v, inter.idx, inter.n_keep, inter.offsets, budget, inter.k_out, inter.v_out, stream)
+        e[4].record(stream)
+    barrier()
+    stage_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / args.steps for i, n in enumerate(names)}
+    clocks = sampler.stop() if sampler else None
+    del inter
+
+    # ---- end to end: pinned host inputs -> device, pass, results -> pinned host
+    e2e = None
+    if not args.no_e2e:
+        hq = [t.cpu().pin_memory() for t in wl.q]
+        hk = [t.cpu().pin_memory() for t in wl.k]
+        hv = [t.cpu().pin_memory() for t in wl.v]
+        h_kout = torch.empty(out.k_out.shape, dtype=out.k_out.dtype).pin_memory()
+        h_vout = torch.empty(out.v_out.shape, dtype=out.v_out.dtype).pin_memory()
+        h_nkeep = torch.empty(out.n_keep.shape, dtype=out.n_keep.dtype).pin_memory()
+        h_off = torch.empty(out.offsets.shape, dtype=out.offsets.dtype).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in hq + hk + hv)
+        d2h = sum(t.numel() * t.element_size() for t in (h_kout, h_vout, h_nkeep, h_off))
+
+        def e2e_step():
+            for l in range(cfg.n_layers):
+                wl.q[l].copy_(hq[l], non_blocking=True)
+                wl.k[l].copy_(hk[l], non_blocking=True)
+                wl.v[l].copy_(hv[l], non_blocking=True)
+            step()
+            h_kout.copy_(out.k_out, non_blocking=True)
+            h_vout.copy_(out.v_out, non_blocking=True)
+            h_nkeep.copy_(out.n_keep, non_blocking=True)
+            h_off.copy_(out.offsets, non_blocking=True)
+
+        e2e_steps = max(3, min(args.steps, 10))
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        f1.record(stream)
+        barrier()
+        e2e_ms = max(f0.elapsed_time(f1), (time.perf_counter() - t0) * 1e3) / e2e_steps
+        assert int(h_nkeep.sum()) == budget * cfg.batch
+        e2e = dict(ms=e2e_ms, h2d=h2d, d2h=d2h, steps=e2e_steps)
+        del hq, hk, hv, h_kout, h_vout
+
+    # ---- max over ranks
+    t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0] + [stage_ms[n] for n in names], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    stage_ms = {n: float(t[2 + i]) for i, n in enumerate(names)}
+
+    if rank == 0:
+        ms_per_step = ms_total / args.steps
+        tokens = cfg.batch * cfg.n_ctx * world
+        value = tokens / (ms_per_step * 1e-3)
+        peak, peak_kind = measured_peaks()
+        ab = algorithmic_bytes(cfg)
+        dominant = max(("score", "gather"), key=lambda n: stage_ms[n])
+        ach = ab[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
+        line = dict(
+            metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+            ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+            dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
+            config=workload_config(cfg, world), clocks=clocks, gpu_launches=int(launches),
+            stage_ms=stage_ms,
+            pass_roofline=dict(bytes=ab["total"], achieved=ab["total"] / (ms_per_step * 1e-3) / 1e9, peak=peak,
+                               unit="GB/s", frac=ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
+                               peak_kind=peak_kind, frac_of_8tbs=ab["total"] / (ms_per_step * 1e-3) / 8e12),
+            roofline=dict(bound="hbm", kernel=dominant, achieved=ach, peak=peak, unit="GB/s", frac=ach / peak,
+                          traffic=None, peak_kind=peak_kind, algorithmic_bytes=ab[dominant]),
+        )
+        if e2e:
+            line["e2e"] = dict(value=tokens / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=e2e["h2d"],
+                               d2h_bytes_per_step=e2e["d2h"], ms_per_step=e2e_ms, steps=e2e["steps"])
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(cfg, args.cpu_seconds)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
