@@ -26,15 +26,22 @@ kvc_status check_cuda(cudaError_t e, const char* what) {
 
 void count_launch(int n) { g_launches += n; }
 
-size_t score_generic_workspace_bytes(const Problem& P);
-kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
-                                const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,
-                                cudaStream_t st);
-
-size_t score_workspace_bytes(const Problem& P) { return score_generic_workspace_bytes(P); }
+size_t score_workspace_bytes(const Problem& P) {
+  size_t a = score_generic_workspace_bytes(P);
+  if (score_sm100_supported(P)) {
+    const size_t b = score_sm100_workspace_bytes(P);
+    if (b > a) a = b;
+  }
+  return a;
+}
 
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
-                        float* scores, void* ws, size_t ws_bytes, cudaStream_t st) {
+                        float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
+  if (score_sm100_supported(P)) {
+    const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st);
+    if (s == KVC_OK) return launch_score_augment(P, scores, st);
+    if (s != KVC_ERR_UNSUPPORTED) return s;      // a real failure; UNSUPPORTED = strides TMA cannot take
+  }
   return launch_score_generic(P, gm, q, k, scores, ws, ws_bytes, st);
 }
 
@@ -236,7 +243,7 @@ kvc_status kvc_score(const kvc_desc* d, const void* const* q, const void* const*
   KVC_REQUIRE(scores != nullptr, KVC_ERR_INVALID_ARG, "scores is NULL");
   if ((s = check_ws(ws, ws_bytes, score_workspace_bytes(P))) != KVC_OK) return s;
   if ((s = check_device()) != KVC_OK) return s;
-  return launch_score(P, gm, qp, kp, scores, ws, ws_bytes, (cudaStream_t)stream);
+  return launch_score(P, gm, qp, kp, scores, nullptr, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 kvc_status kvc_compose(const kvc_desc* d, const float* scores, int32_t* idx, float* composite,
@@ -313,7 +320,7 @@ kvc_status kvc_compress(const kvc_desc* d, const void* const* q, const void* con
   const size_t stage_bytes = lay.alloc - lay.stage;
 
   if (device_status) KVC_CUDA(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
-  if ((s = launch_score(P, gm, qp, kp, scores, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
+  if ((s = launch_score(P, gm, qp, kp, scores, device_status, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
   if ((s = launch_compose(P, scores, idx, composite, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
   if ((s = launch_allocate(P, composite, budget, n_keep, reinterpret_cast<long long*>(offsets),
                            w + lay.alloc, lay.total - lay.alloc, st)) != KVC_OK) return s;

@@ -60,7 +60,18 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 size_t score_workspace_bytes(const Problem& P);
 // Eqs. 3, 14-16: writes scores [L, Bt, Hkv, N].
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
-                        float* scores, void* ws, size_t ws_bytes, cudaStream_t st);
+                        float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
+// The two implementations behind it: CUDA cores (any supported shape) and tcgen05 (bf16, GQA
+// groups of up to 128 window rows).
+size_t score_generic_workspace_bytes(const Problem& P);
+kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
+                                const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,
+                                cudaStream_t st);
+kvc_status launch_score_augment(const Problem& P, float* scores, cudaStream_t st);
+bool score_sm100_supported(const Problem& P);
+size_t score_sm100_workspace_bytes(const Problem& P);
+kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
+                              int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
 
 // ---- rank + compose ---------------------------------------------------------------------------
 size_t compose_workspace_bytes(const Problem& P);
