@@ -46,6 +46,7 @@ def parse_args():
     ap.add_argument("--retention", type=float, default=None)
     ap.add_argument("--n-ctx", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers of the same shape (profiling captures)")
     ap.add_argument("--elem-std", type=float, default=None)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -64,6 +65,9 @@ def pick_config(args):
         kw["n_ctx"] = args.n_ctx
     if args.batch is not None:
         kw["batch"] = args.batch
+    if args.layers is not None:
+        kw["n_layers"] = args.layers
+        kw["name"] = "%s_L%d" % (cfg.name, args.layers)
     if args.elem_std is not None:
         kw["elem_std"] = args.elem_std
     return cfg.replace(**kw) if kw else cfg
