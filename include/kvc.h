@@ -54,6 +54,7 @@ typedef enum { KVC_F32 = 0, KVC_BF16 = 1 } kvc_dtype;
 typedef enum { KVC_AGG_MAX = 0, KVC_AGG_MEAN = 1 } kvc_agg;
 
 #define KVC_MAX_LAYERS 128
+#define KVC_STATIC_MAX_BATCH 64 /* largest batch kvc_allocate_static accepts */
 
 /*
  * Problem description (Sec. 3.1: L layers, K, V in R^{Hkv x N x d}; Sec. 2.2: G = Hq / Hkv).
@@ -141,6 +142,30 @@ KVC_API kvc_status kvc_compose(const kvc_desc* desc, const float* scores, int32_
 KVC_API kvc_status kvc_allocate(const kvc_desc* desc, const float* composite, int64_t budget,
                         int32_t* n_keep, int64_t* offsets, void* workspace,
                         size_t workspace_bytes, void* stream);
+
+/*
+ * kvc_allocate without a workspace argument (the paper has no counterpart to this entry point; it
+ * is kvc_allocate, same inputs, same outputs, same result).
+ *
+ * It is meant for callers that may not allocate device memory and so cannot supply a workspace:
+ * an inference server that plans all of its device memory at start-up and forbids cudaMalloc
+ * afterwards (the call synchronises the device and can fail once memory is fragmented), or a
+ * plug-in that is handed the host application's tensors but no allocator.  The scratch of the
+ * selection lives instead in a fixed array inside the library image: 256 KiB of device memory on
+ * every GPU that loads the library, held until the process exits.  The call allocates and frees
+ * nothing, on the device or through any library.
+ *
+ *   - desc->batch must be <= KVC_STATIC_MAX_BATCH; a larger batch returns KVC_ERR_UNSUPPORTED
+ *     and launches nothing.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps what the last call left in it; each
+ *     call clears the part it uses, in stream order, before its first kernel.  Two calls whose
+ *     work overlaps on the GPU (different streams, no dependency between them) race on it: order
+ *     them, or use kvc_allocate with separate workspaces.
+ */
+KVC_API kvc_status kvc_allocate_static(const kvc_desc* desc, const float* composite, int64_t budget,
+                               int32_t* n_keep, int64_t* offsets, void* stream);
 
 /*
  * Compaction (Eqs. 23-24): K'[l][h, k, :] = K[l][h, idx[l, h, k], :] for k < n_keep[l]; V alike.

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     KvcError,
     desc_from_config,
     kvc_allocate,
+    kvc_allocate_static,
     kvc_budget_from_ratio,
     kvc_compose,
     kvc_compress,

@@ -70,6 +70,8 @@ def _load():
     lib.kvc_compose.restype = C.c_int
     lib.kvc_allocate.argtypes = [dp, vp, i64, vp, vp, vp, sz, vp]
     lib.kvc_allocate.restype = C.c_int
+    lib.kvc_allocate_static.argtypes = [dp, vp, i64, vp, vp, vp]
+    lib.kvc_allocate_static.restype = C.c_int
     lib.kvc_gather.argtypes = [dp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
     lib.kvc_gather.restype = C.c_int
     lib.kvc_compress.argtypes = [dp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -145,6 +147,13 @@ def kvc_allocate(desc, composite, budget, n_keep, offsets, workspace, stream=Non
     wp, wb = _ws(workspace)
     _check(_load().kvc_allocate(C.byref(desc), _dptr(composite), int(budget), _dptr(n_keep),
                                 _dptr(offsets), wp, wb, _stream(stream)))
+
+
+def kvc_allocate_static(desc, composite, budget, n_keep, offsets, stream=None) -> None:
+    """``kvc_allocate`` for callers that cannot allocate a workspace: the scratch is a fixed array
+    inside the library (batch <= 64).  Calls that overlap on the GPU share that array and race."""
+    _check(_load().kvc_allocate_static(C.byref(desc), _dptr(composite), int(budget), _dptr(n_keep),
+                                       _dptr(offsets), _stream(stream)))
 
 
 def kvc_gather(desc, k, v, idx, n_keep, offsets, budget, k_out, v_out, stream=None) -> None:

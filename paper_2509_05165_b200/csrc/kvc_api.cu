@@ -192,6 +192,14 @@ CompressLayout compress_layout(const Problem& P) {
 }
 
 }  // namespace
+
+kvc_status resolve_desc(const kvc_desc* d, Problem* P) {
+  GroupMap gm;
+  return resolve(d, P, &gm);
+}
+kvc_status require_budget(const Problem& P, long long budget) { return check_budget(P, budget); }
+kvc_status require_device() { return check_device(); }
+
 }  // namespace kvc
 
 using namespace kvc;

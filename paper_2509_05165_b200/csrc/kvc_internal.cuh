@@ -53,6 +53,11 @@ void count_launch(int n = 1);
     if (_s != KVC_OK) return _s;                              \
   } while (0)
 
+// Host-side validation shared by the entry points that live outside kvc_api.cu.
+kvc_status resolve_desc(const kvc_desc* d, Problem* P);
+kvc_status require_budget(const Problem& P, long long budget);
+kvc_status require_device();
+
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 // ---- score ------------------------------------------------------------------------------------
