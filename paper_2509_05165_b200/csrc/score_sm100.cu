@@ -3,37 +3,60 @@
 // One persistent kernel, one CTA per SM.  K is streamed from HBM exactly once:
 //
 //   pass 1 (statistics)  tile = 128 tokens.  D[query row, token] = Q K^T on tcgen05 with the
-//                        accumulator in TMEM; every query row keeps a running (max, sum-exp) in
-//                        registers (rows sit on TMEM lanes, so the row reduction is in-thread).
-//   exchange             the partial (max, sum) of the CTAs that shared a (layer, sequence, KV
-//                        head) unit are combined by whichever CTA finishes the unit last, which
-//                        publishes the rows' log-sum-exp and raises the unit's flag.
-//   pass 2 (emit)        runs a fixed number of work items behind pass 1, so its K tiles are still
-//                        in L2.  D[token, query row] = K Q^T (operands swapped: tokens on TMEM
-//                        lanes), so the max over the window rows (Eq. 14) and the mean/max over the
-//                        query heads of the group (Eq. 15) are in-thread and the score store is
-//                        coalesced.  max_m exp(s_m - lse_m) is evaluated as exp(max_m(s_m - lse_m)):
-//                        one exponential per query head, not per row.
+//                        accumulator in TMEM.  Query rows sit on TMEM lanes, so the softmax
+//                        denominator of a row (Eq. 3) is an in-thread sum: every row keeps a
+//                        reference exponent and a running sum of 2^(logit - reference).
+//   exchange             a run of kRunTiles consecutive tiles of one (layer, sequence, KV head)
+//                        unit yields one partial (reference, sum) per row.  A helper warp pushes
+//                        it to global memory and counts it into its group of kGroupRuns runs;
+//                        whichever CTA completes a group hands it to its second helper warp,
+//                        which folds the group's partials (fixed order) and counts the group
+//                        into the unit; whoever completes the unit folds the group results into
+//                        the rows' log-sum-exp.  Both folds are one batch of loads, and neither
+//                        sits on the path of the CTA's own tiles.
+//   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
+//                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
+//                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
+//                        mean/max over the query heads of the group (Eq. 15) are in-thread and
+//                        the score store is coalesced.  max_m exp(s_m - lse_m) is evaluated as
+//                        exp(max_m(s_m - lse_m)): one exponential per query head, not per row.
 //
-// Both passes are interleaved in one static, globally ordered work list that every CTA walks
-// with the same stride; an item of pass 2 only ever waits for items of pass 1 that lie a full
-// round earlier in that order, so the walk cannot deadlock while all CTAs are resident.  Every
-// wait (mbarrier or flag) is bounded; on expiry the kernel records KVC_ERR_TIMEOUT and drains.
+// Every CTA walks one static sequence that alternates a pass-1 tile with a pass-2 tile; the
+// pass-2 stream trails the pass-1 stream by `shift` tiles.  A pass-2 tile only ever waits for
+// pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot deadlock while all
+// CTAs are resident.  Every wait (mbarrier or global flag) is bounded; on expiry the kernel
+// records KVC_ERR_TIMEOUT, stops computing and drains.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 4-7 and 8-11 =
-// two epilogue warpgroups (each takes every other tile and owns two of the four TMEM buffers).
+// Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch), warp 1 = MMA
+// issuer and TMEM owner, warp 2 = statistics push, warp 3 = statistics fold, warps 4-11 = pass-1 epilogue (two
+// warpgroups, each takes one half of every tile's columns), warps 12-15 = pass-2 epilogue.
 #include <cuda.h>
 
 #include "kvc_internal.cuh"
+
+#ifndef KVC_SCORE_RUN_TILES
+#define KVC_SCORE_RUN_TILES 4      // tiles per run
+#endif
+#ifndef KVC_SCORE_LAG_EXTRA
+#define KVC_SCORE_LAG_EXTRA 2      // runs of slack between a unit's last pass-1 run and its first pass-2 run
+#endif
+#ifndef KVC_SCORE_PREFETCH
+#define KVC_SCORE_PREFETCH 4       // pass-1 tiles prefetched into L2 ahead of their load
+#endif
 
 namespace kvc {
 namespace {
 
 constexpr int kTile = 128;            // tokens per tile = MMA M = MMA N
-constexpr int kFastThreads = 384;
-constexpr int kEpiWarp0 = 4;
+constexpr int kFastThreads = 512;
 constexpr int kRows = 128;            // query rows per unit handled by one MMA (R <= 128)
+constexpr int kRunTiles = KVC_SCORE_RUN_TILES;
+constexpr int kGroupRuns = 8;         // runs whose partials are folded together at the first level
+constexpr int kJobSlots = 8;          // fold jobs that may wait in the CTA's queue
+constexpr int kQSlots = 3;
+constexpr int kPrefetch = KVC_SCORE_PREFETCH;
 constexpr float kLog2eF = 1.4426950408889634f;
+constexpr float kRescaleLimit = 1.8446744e19f;               // 2^64: a chunk sum beyond it restarts with a new reference
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
 
 constexpr int kMaxFastLayers = 112;   // 2 tensor maps per layer must fit the 32 KB kernel-parameter space
@@ -41,16 +64,18 @@ constexpr int kMaxFastLayers = 112;   // 2 tensor maps per layer must fit the 32
 struct FastParams {
   CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (d, N, Hkv, Bt), box 64 x 128 x 1 x 1, 128-byte swizzle
   CUtensorMap q_maps[kMaxFastLayers];   // Q^(l) as (d, w, Hq, Bt), box 64 x w x G x 1
-  float2* partial;             // [U][NS][2][128]
-  float* lse2;                 // [U][128]
-  int* counter;                // [U]
-  int* flag;                   // [U]
+  float4* partial;             // [U][RPU][32 lanes][2]: (ref, sum) of rows 4i .. 4i+3 of one run
+  float4* group_partial;       // [U][NG][32 lanes][2]: the same, folded over a group of runs
+  int* group_counter;          // [U][NG], preset to -1
+  int* unit_counter;           // [U], preset to -1
+  unsigned int* lse2;          // [U][128] fp32 bits, preset to 0xffffffff ("not there yet")
   int* status;                 // device status word (may be null)
   float* scores;               // [U][N]
   int L, Bt, Hkv, G, R;
   long long N, q_pos0;
-  int U, C, NT, RUN, LAG, NS;  // units, items per unit, tiles per unit, run length, lag, partial slots
-  long long E;                 // number of list entries = U * C + LAG
+  int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
+  unsigned int total_runs;     // U * RPU
+  long long shift;             // tiles by which the pass-2 stream trails the pass-1 stream
   float sl2e;                  // scale * log2(e)
   int agg_group;
 };
@@ -98,10 +123,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c0, int c1, int c2, int c3) {
+                                            int c0, int c1, int c2, int c3, unsigned long long policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -116,8 +146,8 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 consecutive accumulator columns of this thread's TMEM lane; the caller waits for the load.
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -127,25 +157,57 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two fp32 lanes in one 64-bit register (Blackwell packed fp32 arithmetic).
+__device__ __forceinline__ unsigned long long pack2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long pack2u(uint32_t a, uint32_t b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long p, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(p));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void named_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const unsigned int* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(int* p, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_relaxed_u32(unsigned int* p, uint32_t v) {
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart,
@@ -163,38 +225,42 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t addr) {
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) |
                             ((uint32_t)(kTile >> 4) << 24);
 
-// ------------------------------------------------------------------------------------------------
-// Work list
-// ------------------------------------------------------------------------------------------------
-struct Entry {
-  bool has1, has2;
-  int u1, ch1, u2, ch2;
-};
-__device__ __forceinline__ Entry decode(const FastParams& P, long long e) {
-  Entry t;
-  const long long n1 = (long long)P.U * P.C;
-  t.has1 = e < n1;
-  t.u1 = t.has1 ? (int)(e / P.C) : -1;
-  t.ch1 = t.has1 ? (int)(e - (long long)t.u1 * P.C) : 0;
-  const long long p = e - P.LAG;
-  t.has2 = p >= 0 && p < n1;
-  t.u2 = t.has2 ? (int)(p / P.C) : -1;
-  t.ch2 = t.has2 ? (int)(p - (long long)t.u2 * P.C) : 0;
-  return t;
+// (reference, sum) pairs of the same row: fold (m, l) into (M, Ls).  Exponents are base 2.
+__device__ __forceinline__ void combine(float& M, float& Ls, float m, float l) {
+  const float Mn = fmaxf(M, m);
+  if (Mn > -INFINITY) Ls = Ls * ex2(M - Mn) + l * ex2(m - Mn);
+  M = Mn;
 }
-// Next list entry of this CTA after e (runs of RUN consecutive entries, stride gridDim.x runs).
-__device__ __forceinline__ long long next_entry(const FastParams& P, long long e) {
-  const long long r = e / P.RUN;
-  const int k = (int)(e - r * P.RUN);
-  if (k + 1 < P.RUN && e + 1 < P.E) return e + 1;
-  const long long e2 = (r + gridDim.x) * P.RUN;
-  return e2 < P.E ? e2 : -1;
+
+// ------------------------------------------------------------------------------------------------
+// The static per-CTA sequence.  Stream position idx -> (run ordinal, tile); a run is kRunTiles
+// consecutive tiles of one unit, runs are dealt to the CTAs round-robin.
+// ------------------------------------------------------------------------------------------------
+struct TileRef {
+  bool valid;
+  int t;        // position inside the run
+  int u;        // unit = (layer, sequence, KV head)
+  int j;        // run inside the unit
+  int tile;     // tile inside the unit
+  bool last;    // last valid tile of its run
+};
+__device__ __forceinline__ TileRef decode(const FastParams& P, long long idx) {
+  TileRef r;
+  const unsigned int k = (unsigned int)idx / kRunTiles;      // the host keeps every index below 2^31
+  r.t = (int)((unsigned int)idx - k * kRunTiles);
+  const unsigned int run = blockIdx.x + k * (unsigned int)P.grid;
+  r.u = (int)(run / (unsigned int)P.RPU);
+  r.j = (int)(run - (unsigned int)r.u * (unsigned int)P.RPU);
+  r.tile = r.j * kRunTiles + r.t;
+  r.valid = r.tile < P.NT;
+  r.last = r.valid && (r.t == kRunTiles - 1 || r.tile + 1 >= P.NT);
+  return r;
 }
 __device__ __forceinline__ void unit_coords(const FastParams& P, int u, int* l, int* b, int* h) {
-  *h = u % P.Hkv;
-  const int lb = u / P.Hkv;
-  *b = lb % P.Bt;
-  *l = lb / P.Bt;
+  const unsigned int lb = (unsigned int)u / (unsigned int)P.Hkv;
+  *h = (int)((unsigned int)u - lb * (unsigned int)P.Hkv);
+  *l = (int)(lb / (unsigned int)P.Bt);
+  *b = (int)(lb - (unsigned int)*l * (unsigned int)P.Bt);
 }
 
 template <int D>
@@ -202,22 +268,26 @@ struct SmemLayout {
   static constexpr int kHalves = D / 64;
   static constexpr int kTileBytes = kTile * D * 2;
   static constexpr int kStages = (D == 128) ? 4 : 8;
-  static constexpr int kQ = 0;                                 // two Q buffers
-  static constexpr int kK = 2 * kTileBytes;                    // K stage ring
+  static constexpr int kQ = 0;                                 // Q ring
+  static constexpr int kK = kQSlots * kTileBytes;              // K stage ring
   static constexpr int kMisc = kK + kStages * kTileBytes;
-  // misc: barriers then small arrays
-  static constexpr int kBarFull = kMisc;                       // kStages x 8
-  static constexpr int kBarEmpty = kBarFull + 8 * kStages;
-  static constexpr int kBarTFull = kBarEmpty + 8 * kStages;    // 4 x 8
+  static constexpr int kBarKFull = kMisc;                      // kStages x 8
+  static constexpr int kBarKEmpty = kBarKFull + 8 * kStages;
+  static constexpr int kBarTFull = kBarKEmpty + 8 * kStages;   // 4 x 8
   static constexpr int kBarTEmpty = kBarTFull + 32;
-  static constexpr int kBarQFull = kBarTEmpty + 32;            // 2 x 8
-  static constexpr int kBarQFree = kBarQFull + 16;
-  static constexpr int kTmemSlot = kBarQFree + 16;             // 4 B (+ padding)
+  static constexpr int kBarQFull = kBarTEmpty + 32;            // kQSlots x 8
+  static constexpr int kBarQFree = kBarQFull + 8 * kQSlots;
+  static constexpr int kBarSFull = kBarQFree + 8 * kQSlots;    // statistics stage: full / empty
+  static constexpr int kBarSEmpty = kBarSFull + 8;
+  static constexpr int kTmemSlot = kBarSEmpty + 8;             // 4 B (+ padding)
   static constexpr int kAbort = kTmemSlot + 8;                 // 4 B
-  static constexpr int kBcast = kAbort + 8;                    // 2 x 4 B
-  static constexpr int kLse = kBcast + 16;                     // 2 x 128 floats
-  static constexpr int kTotal = kLse + 2 * kRows * 4;
-  static constexpr int kDynamic = kTotal + 1024;               // slack for 1024-byte alignment
+  static constexpr int kJobHead = kAbort + 8;                  // 4 B: fold jobs pushed
+  static constexpr int kJobTail = kJobHead + 4;                // 4 B: fold jobs taken
+  static constexpr int kJobs = kJobTail + 4;                   // kJobSlots x 4 B
+  static constexpr int kNegLse = (kJobs + 4 * kJobSlots + 15) / 16 * 16;  // 128 floats, read as 16-byte vectors: -log-sum-exp of the pass-2 unit
+  static constexpr int kStats = kNegLse + kRows * 4;           // 2 halves x 128 rows x float2
+  static constexpr int kTotal = kStats + 2 * kRows * 8;
+  static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -227,25 +297,34 @@ template <int D, int W, bool kTaskMean>
 __global__ void __launch_bounds__(kFastThreads, 1)
 score_sm100_kernel(const __grid_constant__ FastParams P) {
   using SL = SmemLayout<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_word = reinterpret_cast<volatile int*>(smem + SL::kAbort);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SL::kTmemSlot);
 
-  auto bar_full = [&](int s) { return sbase + SL::kBarFull + 8 * s; };
-  auto bar_empty = [&](int s) { return sbase + SL::kBarEmpty + 8 * s; };
+  if ((sbase & 1023u) != 0) {          // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0 && P.status) atomicCAS(P.status, 0, (int)KVC_ERR_CUDA);
+    return;
+  }
+
+  auto bar_kfull = [&](int s) { return sbase + SL::kBarKFull + 8 * s; };
+  auto bar_kempty = [&](int s) { return sbase + SL::kBarKEmpty + 8 * s; };
   auto bar_tfull = [&](int b) { return sbase + SL::kBarTFull + 8 * b; };
   auto bar_tempty = [&](int b) { return sbase + SL::kBarTEmpty + 8 * b; };
   auto bar_qfull = [&](int q) { return sbase + SL::kBarQFull + 8 * q; };
   auto bar_qfree = [&](int q) { return sbase + SL::kBarQFree + 8 * q; };
+  const uint32_t bar_sfull = sbase + SL::kBarSFull, bar_sempty = sbase + SL::kBarSEmpty;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < SL::kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-    for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), 4); }
-    for (int q = 0; q < 2; ++q) { mbar_init(bar_qfull(q), 1); mbar_init(bar_qfree(q), 1); }
+    for (int s = 0; s < SL::kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
+    for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), b < 2 ? 8 : 4); }
+    for (int q = 0; q < kQSlots; ++q) { mbar_init(bar_qfull(q), 1); mbar_init(bar_qfree(q), 1); }
+    mbar_init(bar_sfull, 8);
+    mbar_init(bar_sempty, 1);
     *abort_word = 0;
+    *reinterpret_cast<volatile int*>(smem + SL::kJobHead) = 0;
+    *reinterpret_cast<volatile int*>(smem + SL::kJobTail) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -258,291 +337,432 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // this CTA's share of the runs and the length of its sequence
+  const long long my_runs = (P.total_runs > blockIdx.x) ? (P.total_runs - blockIdx.x + P.grid - 1) / P.grid : 0;
+  const long long my_tiles = my_runs * kRunTiles;            // stream length (some positions hold no tile)
+  const long long n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
   const uint32_t q_bytes = (uint32_t)P.R * D * 2;
+  const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
   if (warp == 0) {
     // ============================== TMA producer ==============================================
     if (lane == 0) {
-      long long n = 0;                 // tiles issued so far
-      int cur_u[2] = {-1, -1};
-      uint32_t qfree_phase[2] = {0, 0};
+      unsigned long long pol_stream, pol_keep;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+      long long nk = 0;                // K tiles issued
+      long long qc = 0;                // Q tiles issued
       bool ok = true;
-      for (long long e = (long long)blockIdx.x * P.RUN; e >= 0 && e < P.E && ok; e = next_entry(P, e)) {
-        const Entry t = decode(P, e);
-        for (int part = 0; part < 2 && ok; ++part) {
-          if (!(part == 0 ? t.has1 : t.has2)) continue;
-          const int u = part == 0 ? t.u1 : t.u2;
-          const int ch = part == 0 ? t.ch1 : t.ch2;
+      auto prefetch = [&](long long idx) {
+        if (idx >= my_tiles) return;
+        const TileRef t = decode(P, idx);
+        if (!t.valid) return;
+        int l, b, h;
+        unit_coords(P, t.u, &l, &b, &h);
+        for (int hf = 0; hf < SL::kHalves; ++hf) tma_prefetch_4d(P.k_maps + l, hf * 64, t.tile * kTile, h, b);
+      };
+      for (int i = 0; i < kPrefetch; ++i) prefetch(i);
+      for (long long i = 0; i < n_steps && ok; ++i) {
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          const long long idx = pass == 0 ? i : i - P.shift;
+          if (idx < 0 || idx >= my_tiles) continue;
+          const TileRef t = decode(P, idx);
+          if (!t.valid) continue;
           int l, b, h;
-          unit_coords(P, u, &l, &b, &h);
-          if (u != cur_u[part]) {
-            if (cur_u[part] >= 0) {           // the MMAs that read the old Q must have completed
-              ok = mbar_wait(bar_qfree(part), qfree_phase[part], abort_word);
-              qfree_phase[part] ^= 1;
+          unit_coords(P, t.u, &l, &b, &h);
+          if (t.t == 0) {                                    // a new run: its Q goes into the next ring slot
+            const int slot = (int)(qc % kQSlots);
+            if (qc >= kQSlots) {
+              ok = mbar_wait(bar_qfree(slot), (uint32_t)(((qc / kQSlots) - 1) & 1), abort_word);
               if (!ok) break;
             }
-            mbar_expect_tx(bar_qfull(part), q_bytes);
+            mbar_expect_tx(bar_qfull(slot), q_bytes);
             for (int hf = 0; hf < SL::kHalves; ++hf)
-              tma_load_4d(sbase + SL::kQ + part * SL::kTileBytes + hf * (kTile * 128), P.q_maps + l,
-                          bar_qfull(part), hf * 64, 0, h * P.G, b);
-            cur_u[part] = u;
+              tma_load_4d(sbase + SL::kQ + slot * SL::kTileBytes + hf * (kTile * 128), P.q_maps + l,
+                          bar_qfull(slot), hf * 64, 0, h * P.G, b, pol_keep);
+            ++qc;
           }
-          for (int tt = 0; tt < 2; ++tt) {
-            const int tile = 2 * ch + tt;
-            if (tile >= P.NT) break;
-            const int s = (int)(n % SL::kStages);
-            const uint32_t ph = (uint32_t)((n / SL::kStages) & 1);
-            if (n >= SL::kStages) {
-              ok = mbar_wait(bar_empty(s), ph ^ 1, abort_word);
-              if (!ok) break;
-            }
-            mbar_expect_tx(bar_full(s), SL::kTileBytes);
-            for (int hf = 0; hf < SL::kHalves; ++hf)
-              tma_load_4d(sbase + SL::kK + s * SL::kTileBytes + hf * (kTile * 128), P.k_maps + l, bar_full(s),
-                          hf * 64, tile * kTile, h, b);
-            ++n;
+          const int s = (int)(nk % SL::kStages);
+          if (nk >= SL::kStages) {
+            ok = mbar_wait(bar_kempty(s), (uint32_t)(((nk / SL::kStages) - 1) & 1), abort_word);
+            if (!ok) break;
           }
+          mbar_expect_tx(bar_kfull(s), SL::kTileBytes);
+          // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
+          for (int hf = 0; hf < SL::kHalves; ++hf)
+            tma_load_4d(sbase + SL::kK + s * SL::kTileBytes + hf * (kTile * 128), P.k_maps + l, bar_kfull(s),
+                        hf * 64, t.tile * kTile, h, b, pass == 0 ? pol_keep : pol_stream);
+          ++nk;
+          if (pass == 0) prefetch(idx + kPrefetch);
         }
       }
       // drain: every issued copy must have landed before the CTA's shared memory is released
-      const long long first = n > SL::kStages ? n - SL::kStages : 0;
-      for (long long i = first; i < n; ++i)
-        mbar_wait(bar_full((int)(i % SL::kStages)), (uint32_t)((i / SL::kStages) & 1), abort_word);
+      const long long first = nk > SL::kStages ? nk - SL::kStages : 0;
+      for (long long n = first; n < nk; ++n)
+        mbar_wait(bar_kfull((int)(n % SL::kStages)), (uint32_t)((n / SL::kStages) & 1), abort_word);
+      const long long qfirst = qc > kQSlots ? qc - kQSlots : 0;
+      for (long long n = qfirst; n < qc; ++n)
+        mbar_wait(bar_qfull((int)(n % kQSlots)), (uint32_t)((n / kQSlots) & 1), abort_word);
     }
   } else if (warp == 1) {
     // ============================== MMA issuer =================================================
     if (lane == 0) {
-      long long n = 0;
-      long long nw[2] = {0, 0};        // tiles issued per warpgroup
-      int cur_u[2] = {-1, -1};
-      uint32_t qfull_phase[2] = {0, 0};
+      long long nk = 0, qc = 0;
+      long long nt[2] = {0, 0};        // tiles issued per pass
+      int cur_slot[2] = {0, 0};
       bool ok = true;
-      for (long long e = (long long)blockIdx.x * P.RUN; e >= 0 && e < P.E && ok; e = next_entry(P, e)) {
-        const Entry t = decode(P, e);
-        const long long e_next = next_entry(P, e);
-        Entry tn;
-        tn.has1 = tn.has2 = false; tn.u1 = tn.u2 = -1; tn.ch1 = tn.ch2 = 0;
-        if (e_next >= 0) tn = decode(P, e_next);
-        for (int part = 0; part < 2 && ok; ++part) {
-          if (!(part == 0 ? t.has1 : t.has2)) continue;
-          const int u = part == 0 ? t.u1 : t.u2;
-          const int ch = part == 0 ? t.ch1 : t.ch2;
-          if (u != cur_u[part]) {
-            ok = mbar_wait(bar_qfull(part), qfull_phase[part], abort_word);
-            qfull_phase[part] ^= 1;
+      for (long long i = 0; i < n_steps && ok; ++i) {
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          const long long idx = pass == 0 ? i : i - P.shift;
+          if (idx < 0 || idx >= my_tiles) continue;
+          const TileRef t = decode(P, idx);
+          if (!t.valid) continue;
+          if (t.t == 0) {
+            const int slot = (int)(qc % kQSlots);
+            ok = mbar_wait(bar_qfull(slot), (uint32_t)((qc / kQSlots) & 1), abort_word);
             if (!ok) break;
-            cur_u[part] = u;
+            cur_slot[pass] = slot;
+            ++qc;
           }
-          const uint32_t q_addr = sbase + SL::kQ + part * SL::kTileBytes;
-          for (int tt = 0; tt < 2; ++tt) {
-            const int tile = 2 * ch + tt;
-            if (tile >= P.NT) break;
-            const int s = (int)(n % SL::kStages);
-            const int buf = tt * 2 + (int)(nw[tt] & 1);
-            ok = mbar_wait(bar_full(s), (uint32_t)((n / SL::kStages) & 1), abort_word);
-            if (ok && nw[tt] >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(((nw[tt] >> 1) & 1) ^ 1), abort_word);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_addr = sbase + SL::kK + s * SL::kTileBytes;
-            const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
+          const int s = (int)(nk % SL::kStages);
+          const int buf = pass * 2 + (int)(nt[pass] & 1);
+          ok = mbar_wait(bar_kfull(s), (uint32_t)((nk / SL::kStages) & 1), abort_word);
+          if (ok && nt[pass] >= 2)
+            ok = mbar_wait(bar_tempty(buf), (uint32_t)(((nt[pass] >> 1) - 1) & 1), abort_word);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t q_addr = sbase + SL::kQ + cur_slot[pass] * SL::kTileBytes;
+          const uint32_t k_addr = sbase + SL::kK + s * SL::kTileBytes;
+          const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t off = (uint32_t)(kk >> 2) * (kTile * 128) + (uint32_t)(kk & 3) * 32;
-              const uint64_t dq = umma_desc(q_addr + off), dk = umma_desc(k_addr + off);
-              // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
-              if (part == 0) tc_mma_bf16(d_tmem, dq, dk, kIdesc, kk > 0);
-              else tc_mma_bf16(d_tmem, dk, dq, kIdesc, kk > 0);
-            }
-            tc_commit(bar_empty(s));      // the K stage may be refilled once these MMAs are done
-            tc_commit(bar_tfull(buf));    // ... and the accumulator is then complete
-            ++n; ++nw[tt];
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (uint32_t)(kk >> 2) * (kTile * 128) + (uint32_t)(kk & 3) * 32;
+            const uint64_t dq = umma_desc(q_addr + off), dk = umma_desc(k_addr + off);
+            // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
+            if (pass == 0) tc_mma_bf16(d_tmem, dq, dk, kIdesc, kk > 0);
+            else tc_mma_bf16(d_tmem, dk, dq, kIdesc, kk > 0);
           }
-          // release the Q buffer as soon as the last MMA that reads it has been issued
-          const int u_next = part == 0 ? (tn.has1 ? tn.u1 : -1) : (tn.has2 ? tn.u2 : -1);
-          const bool more = e_next >= 0 && (part == 0 ? tn.has1 : tn.has2);
-          if (ok && more && u_next != u) tc_commit(bar_qfree(part));
+          tc_commit(bar_kempty(s));      // the K stage may be refilled once these MMAs are done
+          tc_commit(bar_tfull(buf));     // ... and the accumulator is then complete
+          if (t.last) tc_commit(bar_qfree(cur_slot[pass]));
+          ++nk; ++nt[pass];
         }
       }
     }
-  } else if (warp >= kEpiWarp0) {
-    // ============================== epilogue warpgroups ========================================
-    const int wg = (warp - kEpiWarp0) >> 2;          // 0 or 1: takes tile 2*ch + wg of every item
-    const int quarter = warp & 3;                    // TMEM lane quarter this warp may read
-    const int row = quarter * 32 + lane;             // TMEM lane = query row (pass 1) or token (pass 2)
-    const int wtid = threadIdx.x - (kEpiWarp0 + 4 * wg) * 32;   // 0..127 within the warpgroup
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    int* bcast = reinterpret_cast<int*>(smem + SL::kBcast) + wg;
-    float* lse_s = reinterpret_cast<float*>(smem + SL::kLse) + wg * kRows;
-    const int bar_id = 1 + wg;
-
-    long long nwg = 0;               // tiles consumed by this warpgroup
-    int acc_u = -1;                  // unit whose statistics are being accumulated
-    long long acc_run = 0;
-    float m_run = -INFINITY, l_run = 0.f;
-    int lse_u = -1;
-    bool ok = true;
-
-    // flush the running statistics of (acc_u, acc_run) and, if this was the unit's last part,
-    // reduce all parts to the rows' log-sum-exp and raise the unit's flag
-    auto flush = [&]() {
-      const int u = acc_u;
-      const long long r_first = ((long long)u * P.C) / P.RUN;
-      const long long r_last = ((long long)(u + 1) * P.C - 1) / P.RUN;
-      const int slot = (int)(acc_run - r_first);
-      P.partial[(((long long)u * P.NS + slot) * 2 + wg) * kRows + wtid] = make_float2(m_run, l_run);
-      __threadfence();
-      named_bar(bar_id, 128);
-      if (wtid == 0) {
-        const int expected = 2 * (int)(r_last - r_first + 1);
-        const int old = atomicAdd(P.counter + u, 1);
-        *bcast = (old == expected - 1) ? 1 : 0;
-      }
-      named_bar(bar_id, 128);
-      if (*bcast) {
-        __threadfence();
-        const int nparts = 2 * (int)(r_last - r_first + 1);
-        const float2* p = P.partial + ((long long)u * P.NS * 2) * kRows + wtid;
-        float M = -INFINITY, Ls = 0.f;
-        for (int i = 0; i < nparts; ++i) {
-          const float2 v = __ldcg(p + (long long)i * kRows);
-          const float Mn = fmaxf(M, v.x);
-          if (Mn > -INFINITY) Ls = Ls * ex2(M - Mn) + v.y * ex2(v.x - Mn);
-          M = Mn;
+  } else if (warp < 4) {
+    // ============================== statistics exchange ========================================
+    // Lane i owns rows 4i .. 4i+3.  A (reference, sum) record of 128 rows is 32 lanes x 2 float4.
+    volatile int* job_head = reinterpret_cast<volatile int*>(smem + SL::kJobHead);
+    volatile int* job_tail = reinterpret_cast<volatile int*>(smem + SL::kJobTail);
+    volatile int* jobs = reinterpret_cast<volatile int*>(smem + SL::kJobs);
+    if (warp == 2) {
+      // ---- push: one record per run, counted into its group; a completed group becomes a fold job
+      const float4* stage4 = reinterpret_cast<const float4*>(smem + SL::kStats);   // two rows per float4
+      int head = 0;
+      bool ok = true;
+      auto push_job = [&](int job) {                          // lane 0 only
+        const unsigned long long t0 = globaltimer_ns();
+        while (ok && head - *job_tail >= kJobSlots) {
+          __nanosleep(64);
+          if (*abort_word) ok = false;
+          else if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; ok = false; }
         }
-        P.lse2[(long long)u * kRows + wtid] = M + log2f(Ls);
-        __threadfence();
-        named_bar(bar_id, 128);
-        if (wtid == 0) st_release(P.flag + u, 1);
+        jobs[head % kJobSlots] = job;
+        __threadfence_block();
+        *job_head = ++head;
+      };
+      for (long long k = 0; k < my_runs; ++k) {
+        const unsigned int run = blockIdx.x + (unsigned int)k * (unsigned int)P.grid;
+        const int u = (int)(run / (unsigned int)P.RPU);
+        const int j = (int)(run - (unsigned int)u * (unsigned int)P.RPU);
+        if (ok) ok = mbar_wait(bar_sfull, (uint32_t)(k & 1), abort_word);
+        float4 lo, hi;
+        {
+          const float4 a0 = stage4[2 * lane], a1 = stage4[2 * lane + 1];                       // tokens 0..63
+          const float4 b0 = stage4[kRows / 2 + 2 * lane], b1 = stage4[kRows / 2 + 2 * lane + 1];   // tokens 64..127
+          lo = a0; hi = a1;
+          combine(lo.x, lo.y, b0.x, b0.y);
+          combine(lo.z, lo.w, b0.z, b0.w);
+          combine(hi.x, hi.y, b1.x, b1.y);
+          combine(hi.z, hi.w, b1.z, b1.w);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_sempty);               // the stage may be overwritten
+        float4* dst = P.partial + (((long long)u * P.RPU + j) * 32 + lane) * 2;
+        dst[0] = lo;
+        dst[1] = hi;
+        __syncwarp();
+        if (lane == 0 && ok) {
+          const int g = j / kGroupRuns;
+          const int members = min(kGroupRuns, P.RPU - g * kGroupRuns);
+          const int old = atom_add_acq_rel(P.group_counter + (long long)u * P.NG + g, 1);
+          if (old == members - 2) push_job(u * P.NG + g);     // the counter starts at -1
+        }
       }
-      named_bar(bar_id, 128);
-      acc_u = -1;
-      m_run = -INFINITY; l_run = 0.f;
-    };
-
-    for (long long e = (long long)blockIdx.x * P.RUN; e >= 0 && e < P.E; e = next_entry(P, e)) {
-      const Entry t = decode(P, e);
-      const long long run = e / P.RUN;
-      // ---------------- pass 1: statistics ----------------
-      if (t.has1) {
-        if (acc_u >= 0 && (acc_u != t.u1 || acc_run != run)) flush();
-        if (acc_u < 0) { acc_u = t.u1; acc_run = run; }
-        const int tile = 2 * t.ch1 + wg;
-        if (tile < P.NT) {
-          const int buf = wg * 2 + (int)(nwg & 1);
-          if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((nwg >> 1) & 1), abort_word);
-          tc_fence_after();
-          const long long c0 = (long long)tile * kTile;
-          const long long last_vis = min(P.N - 1, P.q_pos0 + (row % W));   // last visible key of this row
-          const bool full_tile = (c0 + kTile - 1 <= min(P.N - 1, P.q_pos0)); // no masking anywhere in the tile
-#pragma unroll 1
-          for (int j = 0; j < kTile / 32; ++j) {
-            float v[32];
-            tc_ld32(lane_addr + (uint32_t)buf * kTile + j * 32, v);
-            if (ok) {
-              if (!full_tile) {
+      if (lane == 0) push_job(-1);                            // no more jobs
+    } else {
+      // ---- fold: a group's records into one, and the last group of a unit into the log-sum-exp
+      int tail = 0;                                           // kept by lane 0
+      for (;;) {
+        int job = 0;
+        if (lane == 0) {
+          const unsigned long long t0 = globaltimer_ns();
+          while (*job_head == tail) {
+            __nanosleep(128);
+            if (*abort_word) { job = -1; break; }
+            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; job = -1; break; }
+          }
+          if (job == 0) {
+            job = jobs[tail % kJobSlots];
+            *job_tail = ++tail;
+          }
+        }
+        job = __shfl_sync(0xffffffffu, job, 0);
+        if (job < 0) break;
+        __threadfence();                                      // the records were published before the counts we saw
+        const int u = job / P.NG, g = job - u * P.NG;
+        const int members = min(kGroupRuns, P.RPU - g * kGroupRuns);
+        float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
+        {
+          const float4* src = P.partial + (((long long)u * P.RPU + g * kGroupRuns) * 32 + lane) * 2;
+          float4 v[2 * kGroupRuns];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (c0 + j * 32 + i > last_vis) v[i] = -INFINITY;
-              }
-              float x0 = v[0], x1 = v[1], x2 = v[2], x3 = v[3];
+          for (int r = 0; r < kGroupRuns; ++r) {
+            if (r < members) { v[2 * r] = __ldcg(src + r * 64); v[2 * r + 1] = __ldcg(src + r * 64 + 1); }
+          }
 #pragma unroll
-              for (int i = 4; i < 32; i += 4) {
-                x0 = fmaxf(x0, v[i + 0]); x1 = fmaxf(x1, v[i + 1]);
-                x2 = fmaxf(x2, v[i + 2]); x3 = fmaxf(x3, v[i + 3]);
-              }
-              const float cmax = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-              const float m_new = fmaxf(m_run, cmax * P.sl2e);
-              if (m_new > -INFINITY) {
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  a0 += ex2(fmaf(v[i + 0], P.sl2e, -m_new));
-                  a1 += ex2(fmaf(v[i + 1], P.sl2e, -m_new));
-                  a2 += ex2(fmaf(v[i + 2], P.sl2e, -m_new));
-                  a3 += ex2(fmaf(v[i + 3], P.sl2e, -m_new));
-                }
-                l_run = l_run * ex2(m_run - m_new) + ((a0 + a1) + (a2 + a3));
-                m_run = m_new;
-              }
+          for (int r = 0; r < kGroupRuns; ++r) {
+            if (r < members) {
+              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
+              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
+              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
+              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
             }
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tempty(buf));
-          ++nwg;
+        }
+        float4* dst = P.group_partial + ((long long)job * 32 + lane) * 2;
+        dst[0] = lo;
+        dst[1] = hi;
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = (atom_add_acq_rel(P.unit_counter + u, 1) == P.NG - 2) ? 1 : 0;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          __threadfence();
+          const float4* src = P.group_partial + ((long long)u * P.NG * 32 + lane) * 2;
+          lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f); hi = lo;
+#pragma unroll 4
+          for (int r = 0; r < P.NG; ++r) {
+            const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
+            combine(lo.x, lo.y, v0.x, v0.y);
+            combine(lo.z, lo.w, v0.z, v0.w);
+            combine(hi.x, hi.y, v1.x, v1.y);
+            combine(hi.z, hi.w, v1.z, v1.w);
+          }
+          unsigned int* out = P.lse2 + (long long)u * kRows + 4 * lane;
+          st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
+          st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
+          st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
+          st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
         }
       }
-      // flush at the end of a run (the next entry of this CTA lies in another run) or of pass 1
-      if (acc_u >= 0) {
-        const long long e_next = next_entry(P, e);
-        const bool run_ends = e_next < 0 || e_next / P.RUN != run || !(e_next < (long long)P.U * P.C);
-        if (run_ends) flush();
+    }
+  } else if (warp < 12) {
+    // ============================== pass-1 epilogue ============================================
+    const int half = (warp - 4) >> 2;                 // which 64 columns (tokens) of every tile
+    const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
+    const int row = quarter * 32 + lane;              // TMEM lane = query row
+    const bool row_used = row < P.R;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + half * kRows + row;
+    const long long row_vis = min(P.N - 1, P.q_pos0 + (row % W));     // last key this row sees
+    const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
+
+    long long n1 = 0, runs_done = 0;
+    float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
+    bool ok = true;
+
+    // 32 logits with masking and a reference that follows the maximum
+    auto slow_chunk = [&](const uint32_t (&r)[32], long long c_first, bool masked) {
+      float v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        v[i] = __uint_as_float(r[i]);
+        if (masked && c_first + i > row_vis) v[i] = -INFINITY;
       }
-      // ---------------- pass 2: emit ----------------
-      if (t.has2) {
-        if (lse_u != t.u2) {
-          if (wtid == 0 && ok) {
+      float x0 = v[0], x1 = v[1];
+#pragma unroll
+      for (int i = 2; i < 32; i += 2) { x0 = max3(x0, v[i], v[i + 1]); }
+      const float m_new = fmaxf(mref, fmaxf(x0, x1) * P.sl2e);
+      if (m_new > -INFINITY) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          a0 += ex2(fmaf(v[i + 0], P.sl2e, -m_new));
+          a1 += ex2(fmaf(v[i + 1], P.sl2e, -m_new));
+          a2 += ex2(fmaf(v[i + 2], P.sl2e, -m_new));
+          a3 += ex2(fmaf(v[i + 3], P.sl2e, -m_new));
+        }
+        lsum = lsum * ex2(mref - m_new) + ((a0 + a1) + (a2 + a3));
+        mref = m_new;
+      }
+    };
+    // 32 unmasked logits against the current reference: no maximum, packed arithmetic
+    auto fast_chunk = [&](const uint32_t (&r)[32], long long c_first) {
+      if (mref == -INFINITY) { slow_chunk(r, c_first, false); return; }
+      const unsigned long long neg_ref = pack2(-mref, -mref);
+      unsigned long long acc0 = 0ull, acc1 = 0ull;      // +0.0f twice
+#pragma unroll
+      for (int i = 0; i < 32; i += 4) {
+        const unsigned long long y0 = fma2(pack2u(r[i], r[i + 1]), scale2, neg_ref);
+        const unsigned long long y1 = fma2(pack2u(r[i + 2], r[i + 3]), scale2, neg_ref);
+        float a, b, c, d;
+        unpack2(y0, a, b);
+        unpack2(y1, c, d);
+        acc0 = add2(acc0, pack2(ex2(a), ex2(b)));
+        acc1 = add2(acc1, pack2(ex2(c), ex2(d)));
+      }
+      float s0, s1, s2, s3;
+      unpack2(acc0, s0, s1);
+      unpack2(acc1, s2, s3);
+      const float s = (s0 + s1) + (s2 + s3);
+      if (s < kRescaleLimit) lsum += s;                 // also false for inf / NaN
+      else slow_chunk(r, c_first, false);               // a logit far above the reference: move it
+    };
+
+    for (long long idx = 0; idx < my_tiles; ++idx) {
+      const TileRef t = decode(P, idx);
+      if (!t.valid) continue;
+      const int buf = (int)(n1 & 1);
+      if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word);
+      tc_fence_after();
+      const long long c0 = (long long)t.tile * kTile + half * 64;
+      const bool full = (long long)t.tile * kTile + kTile - 1 <= vis_all;     // no masking anywhere in the tile
+      uint32_t ra[32], rb[32];
+      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64, ra);
+      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64 + 32, rb);
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty(buf));      // the accumulator is in registers now
+      ++n1;
+      if (ok && row_used) {
+        if (full) {
+          fast_chunk(ra, c0);
+          fast_chunk(rb, c0 + 32);
+        } else {
+          slow_chunk(ra, c0, true);
+          slow_chunk(rb, c0 + 32, true);
+        }
+      }
+      if (t.last) {
+        // hand the run's (reference, sum) to the exchange warps
+        if (ok && runs_done >= 1) ok = mbar_wait(bar_sempty, (uint32_t)((runs_done - 1) & 1), abort_word);
+        *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_sfull);
+        ++runs_done;
+        mref = -INFINITY; lsum = 0.f;
+      }
+    }
+  } else {
+    // ============================== pass-2 epilogue ============================================
+    const int quarter = warp & 3;
+    const int trow = quarter * 32 + lane;             // TMEM lane = token inside the tile; also 0..127 in the group
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    float* neg_lse = reinterpret_cast<float*>(smem + SL::kNegLse);
+    const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
+    const int n_chunks = (P.R + 31) / 32;
+    long long n2 = 0;
+    bool ok = true;
+
+    for (long long idx = 0; idx < my_tiles; ++idx) {
+      const TileRef t = decode(P, idx);
+      if (!t.valid) continue;
+      if (t.t == 0) {
+        // a new run: wait for its unit's log-sum-exp (the value itself is the flag)
+        uint32_t bits = 0xffffffffu;
+        if (ok && trow < P.R) {
+          const unsigned int* src = P.lse2 + (long long)t.u * kRows + trow;
+          bits = ld_relaxed_u32(src);
+          if (bits == 0xffffffffu) {
             const unsigned long long t0 = globaltimer_ns();
             uint32_t spins = 0;
-            while (ld_acquire(P.flag + t.u2) == 0) {
-              __nanosleep(64);
+            while ((bits = ld_relaxed_u32(src)) == 0xffffffffu) {
+              __nanosleep(100);
               if ((++spins & 255u) == 0) {
                 if (*abort_word) break;
                 if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
               }
             }
           }
-          named_bar(bar_id, 128);
-          lse_s[wtid] = __ldcg(P.lse2 + (long long)t.u2 * kRows + wtid);
-          named_bar(bar_id, 128);
-          lse_u = t.u2;
-          if (*abort_word) ok = false;
         }
-        const int tile = 2 * t.ch2 + wg;
-        if (tile < P.NT) {
-          const int buf = wg * 2 + (int)(nwg & 1);
-          if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((nwg >> 1) & 1), abort_word);
-          tc_fence_after();
-          const long long c = (long long)tile * kTile + row;          // this thread's token
-          const bool full_tile = ((long long)tile * kTile + kTile - 1 <= P.q_pos0);
-          const long long m_min = c - P.q_pos0;                       // rows m >= m_min see token c
-          float gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
-          float hacc = kTaskMean ? 0.f : -INFINITY;
+        named_bar(1, 128);                             // everyone is done with the previous unit's values
+        neg_lse[trow] = (trow < P.R) ? -__uint_as_float(bits) : 0.f;
+        named_bar(1, 128);
+        if (*abort_word) ok = false;
+      }
+      const int buf = 2 + (int)(n2 & 1);
+      if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), abort_word);
+      tc_fence_after();
+      const long long c = (long long)t.tile * kTile + trow;          // this thread's token
+      const bool full = (long long)t.tile * kTile + kTile - 1 <= vis_all;
+      const long long m_min = c - P.q_pos0;                           // rows m >= m_min see token c
+      float gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
+      float hacc = kTaskMean ? 0.f : -INFINITY;
+      uint32_t r[32];
+      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile, r);
 #pragma unroll 1
-          for (int j = 0; j < kTile / 32; ++j) {
-            if (j * 32 >= P.R) break;
-            float v[32];
-            tc_ld32(lane_addr + (uint32_t)buf * kTile + j * 32, v);
-            const float4* l4 = reinterpret_cast<const float4*>(lse_s + j * 32);
+      for (int j = 0; j < n_chunks; ++j) {
+        tc_wait_ld();
+        float x[32];
+        {
+          const ulonglong2* l2 = reinterpret_cast<const ulonglong2*>(neg_lse + j * 32);
 #pragma unroll
-            for (int i4 = 0; i4 < 8; ++i4) {
-              const float4 lv = l4[i4];
-              const float lsv[4] = {lv.x, lv.y, lv.z, lv.w};
+          for (int i = 0; i < 8; ++i) {
+            const ulonglong2 nl = l2[i];
+            const unsigned long long y0 = fma2(pack2u(r[4 * i], r[4 * i + 1]), scale2, nl.x);
+            const unsigned long long y1 = fma2(pack2u(r[4 * i + 2], r[4 * i + 3]), scale2, nl.y);
+            unpack2(y0, x[4 * i], x[4 * i + 1]);                     // log2 of the attention weights
+            unpack2(y1, x[4 * i + 2], x[4 * i + 3]);
+          }
+        }
+        if (j + 1 < n_chunks) tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + (j + 1) * 32, r);
+        if (!kTaskMean && full && W >= 32) {
+          // the whole chunk belongs to one query head
+          float a = x[0], b = x[1];
 #pragma unroll
-              for (int ii = 0; ii < 4; ++ii) {
-                const int i = i4 * 4 + ii;
-                const int col = j * 32 + i;
-                float x = fmaf(v[i], P.sl2e, -lsv[ii]);               // log2 of the attention weight
-                if (!full_tile && (col % W) < m_min) x = -INFINITY;
-                if (kTaskMean) hacc += ex2(x); else hacc = fmaxf(hacc, x);
-                if ((col + 1) % W == 0) {                              // a query head is complete
-                  if (col < P.R) {
-                    const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
-                    gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
-                  }
-                  hacc = kTaskMean ? 0.f : -INFINITY;
-                }
+          for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
+          hacc = max3(hacc, a, b);
+          hacc = max3(hacc, x[30], x[31]);
+          if (((j + 1) * 32) % W == 0) {
+            const float s_task = ex2(hacc);
+            gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+            hacc = -INFINITY;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int col = j * 32 + i;
+            float xi = x[i];
+            if (!full && (col % W) < m_min) xi = -INFINITY;
+            if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
+            if ((col + 1) % W == 0) {                                  // a query head is complete
+              if (col < P.R) {
+                const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
+                gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
               }
+              hacc = kTaskMean ? 0.f : -INFINITY;
             }
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tempty(buf));
-          ++nwg;
-          if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
-          if (ok && c < P.N) P.scores[(long long)t.u2 * P.N + c] = gacc;
         }
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty(buf));
+      ++n2;
+      if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
+      if (ok && c < P.N) P.scores[(long long)t.u * P.N + c] = gacc;
     }
   }
 
@@ -590,28 +810,38 @@ bool encode_map(CUtensorMap* m, const void* base, const long long dims[4], const
 }
 
 struct FastPlan {
-  int U, C, NT, RUN, LAG, NS, grid;
-  size_t off_partial, off_lse, off_counter, off_total;
+  int U, NT, RPU, NG, grid;
+  long long total_runs, shift;
+  size_t off_partial, off_group, off_sync, sync_bytes, off_total;
 };
 
-bool make_plan(const Problem& P, FastPlan* pl) {
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return false;
+// sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
+void make_plan(const Problem& P, int sms, FastPlan* pl) {
   pl->U = P.L * P.Bt * P.Hkv;
   pl->NT = (int)((P.N + kTile - 1) / kTile);
-  pl->C = (pl->NT + 1) / 2;
-  pl->RUN = 4;
-  pl->grid = sms;
-  // pass 2 trails pass 1 by one full round of the grid plus one unit
-  pl->LAG = ((pl->grid * pl->RUN + pl->C + pl->RUN - 1) / pl->RUN) * pl->RUN;
-  pl->NS = (pl->C + pl->RUN - 1) / pl->RUN + 1;
+  pl->RPU = (pl->NT + kRunTiles - 1) / kRunTiles;
+  pl->NG = (pl->RPU + kGroupRuns - 1) / kGroupRuns;
+  pl->total_runs = (long long)pl->U * pl->RPU;
+  pl->grid = sms > 0 ? (int)(pl->total_runs < sms ? pl->total_runs : sms) : 1;
+  // pass 2 of a run starts once every CTA has been through the rest of the run's unit (at most
+  // ceil(RPU / grid) runs later) plus some runs that hide the exchange; half a run staggers the
+  // two streams so that they change runs (and Q tiles) at different moments
+  const long long lag_runs = (pl->RPU + pl->grid - 1) / pl->grid + KVC_SCORE_LAG_EXTRA;
+  pl->shift = lag_runs * kRunTiles + kRunTiles / 2;
   size_t off = 0;
-  pl->off_partial = off; off += align_up((size_t)pl->U * pl->NS * 2 * kRows * sizeof(float2));
-  pl->off_lse = off; off += align_up((size_t)pl->U * kRows * sizeof(float));
-  pl->off_counter = off; off += align_up((size_t)pl->U * 2 * sizeof(int));
+  pl->off_partial = off; off += align_up((size_t)pl->total_runs * 64 * sizeof(float4));
+  pl->off_group = off; off += align_up((size_t)pl->U * pl->NG * 64 * sizeof(float4));
+  pl->off_sync = off;      // [U][NG] group counters, [U] unit counters, [U][128] log-sum-exp slots
+  pl->sync_bytes = ((size_t)pl->U * pl->NG + (size_t)pl->U) * sizeof(int) + (size_t)pl->U * kRows * sizeof(float);
+  off += align_up(pl->sync_bytes);
   pl->off_total = off;
-  return true;
+}
+
+int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return sms;
 }
 
 template <int D, int W, bool M>
@@ -619,10 +849,10 @@ kvc_status launch_t(const FastParams& fp, int grid, cudaStream_t st) {
   using SL = SmemLayout<D>;
   static bool attr_set = false;
   if (!attr_set) {
-    KVC_CUDA(cudaFuncSetAttribute(score_sm100_kernel<D, W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kDynamic));
+    KVC_CUDA(cudaFuncSetAttribute(score_sm100_kernel<D, W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal));
     attr_set = true;
   }
-  score_sm100_kernel<D, W, M><<<grid, kFastThreads, SL::kDynamic, st>>>(fp);
+  score_sm100_kernel<D, W, M><<<grid, kFastThreads, SL::kTotal, st>>>(fp);
   KVC_LAUNCH_CHECK("score_sm100_kernel");
   return KVC_OK;
 }
@@ -647,21 +877,15 @@ bool score_sm100_supported(const Problem& P) {
   if ((long long)G * P.w > kRows) return false;
   if (P.L > kMaxFastLayers || (long long)P.L * P.Bt * P.Hkv > (1 << 24)) return false;
   if (P.N >= (1LL << 30)) return false;
+  FastPlan pl;
+  make_plan(P, 0, &pl);
+  if ((pl.total_runs + 4096) * kRunTiles + pl.shift >= (1LL << 31)) return false;   // 32-bit sequence indices
   return encode_fn() != nullptr;
 }
 
 size_t score_sm100_workspace_bytes(const Problem& P) {
   FastPlan pl;
-  if (!make_plan(P, &pl)) {
-    // no device yet (host-only size query): assume the largest SM count this library targets
-    pl.U = P.L * P.Bt * P.Hkv;
-    pl.NT = (int)((P.N + kTile - 1) / kTile);
-    pl.C = (pl.NT + 1) / 2;
-    pl.RUN = 4;
-    pl.NS = (pl.C + pl.RUN - 1) / pl.RUN + 1;
-    return align_up((size_t)pl.U * pl.NS * 2 * kRows * sizeof(float2)) +
-           align_up((size_t)pl.U * kRows * sizeof(float)) + align_up((size_t)pl.U * 2 * sizeof(int));
-  }
+  make_plan(P, 0, &pl);
   return pl.off_total;
 }
 
@@ -669,8 +893,10 @@ size_t score_sm100_workspace_bytes(const Problem& P) {
 // for these strides; the caller then uses the CUDA-core path.
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
                               int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
+  const int sms = sm_count();
+  if (sms < 1) return KVC_ERR_UNSUPPORTED;
   FastPlan pl;
-  if (!make_plan(P, &pl)) return KVC_ERR_UNSUPPORTED;
+  make_plan(P, sms, &pl);
   if (ws_bytes < pl.off_total) { set_error("score: workspace too small"); return KVC_ERR_WORKSPACE; }
   const int G = P.Hq / P.Hkv;
   static thread_local FastParams fp;
@@ -685,18 +911,20 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
     if (!encode_map(&fp.q_maps[l], q.p[l], qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
   }
   char* w = reinterpret_cast<char*>(ws);
-  KVC_CUDA(cudaMemsetAsync(w + pl.off_counter, 0, (size_t)pl.U * 2 * sizeof(int), st));
+  // counters start at -1 and the log-sum-exp slots at the "not there yet" pattern: all bits set
+  KVC_CUDA(cudaMemsetAsync(w + pl.off_sync, 0xff, pl.sync_bytes, st));
 
-  fp.partial = reinterpret_cast<float2*>(w + pl.off_partial);
-  fp.lse2 = reinterpret_cast<float*>(w + pl.off_lse);
-  fp.counter = reinterpret_cast<int*>(w + pl.off_counter);
-  fp.flag = fp.counter + pl.U;
+  fp.partial = reinterpret_cast<float4*>(w + pl.off_partial);
+  fp.group_partial = reinterpret_cast<float4*>(w + pl.off_group);
+  fp.group_counter = reinterpret_cast<int*>(w + pl.off_sync);
+  fp.unit_counter = fp.group_counter + (size_t)pl.U * pl.NG;
+  fp.lse2 = reinterpret_cast<unsigned int*>(fp.unit_counter + pl.U);
   fp.status = device_status;
   fp.scores = scores;
   fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G; fp.R = G * P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
-  fp.U = pl.U; fp.C = pl.C; fp.NT = pl.NT; fp.RUN = pl.RUN; fp.LAG = pl.LAG; fp.NS = pl.NS;
-  fp.E = (long long)pl.U * pl.C + pl.LAG;
+  fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.NG = pl.NG; fp.grid = pl.grid;
+  fp.total_runs = (unsigned int)pl.total_runs; fp.shift = pl.shift;
   fp.sl2e = P.scale * kLog2eF;
   fp.agg_group = P.agg_group;
   const bool mean = P.agg_task == KVC_AGG_MEAN;
