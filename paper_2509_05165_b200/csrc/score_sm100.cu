@@ -7,13 +7,14 @@
 //                        denominator of a row (Eq. 3) is an in-thread sum: every row keeps a
 //                        reference exponent and a running sum of 2^(logit - reference).
 //   exchange             a run of kRunTiles consecutive tiles of one (layer, sequence, KV head)
-//                        unit yields one partial (reference, sum) per row.  A helper warp pushes
-//                        it to global memory and counts it into its group of kGroupRuns runs;
-//                        whichever CTA completes a group hands it to its second helper warp,
-//                        which folds the group's partials (fixed order) and counts the group
-//                        into the unit; whoever completes the unit folds the group results into
-//                        the rows' log-sum-exp.  Both folds are one batch of loads, and neither
-//                        sits on the path of the CTA's own tiles.
+//                        unit yields one record of (reference, sum) per row, which the pass-1
+//                        epilogue writes to global memory and counts into its group of
+//                        kGroupRuns runs.  Every group and every unit has a fixed folding CTA
+//                        (round-robin): its exchange warp waits for the count, folds the group's
+//                        records (fixed order) into one and counts the group into the unit, or
+//                        folds a unit's group records into the rows' log-sum-exp.  Each fold is
+//                        one batch of loads, the folds are spread evenly over the CTAs, and none
+//                        of it sits on the path of the CTA's own tiles.
 //   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
 //                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
 //                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
@@ -27,9 +28,12 @@
 // CTAs are resident.  Every wait (mbarrier or global flag) is bounded; on expiry the kernel
 // records KVC_ERR_TIMEOUT, stops computing and drains.
 //
-// Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch), warp 1 = MMA
-// issuer and TMEM owner, warp 2 = statistics push, warp 3 = statistics fold, warps 4-11 = pass-1 epilogue (two
-// warpgroups, each takes one half of every tile's columns), warps 12-15 = pass-2 epilogue.
+// Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch); warp 1 = MMA
+// issuer of pass 1 and TMEM owner; warp 2 = MMA issuer of pass 2 (two issuers, because the
+// waits, commits and bookkeeping around a tile cost one thread more time than the tile's MMAs
+// take, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-11 =
+// pass-1 epilogue (two warpgroups, each takes one half of every tile's columns); warps 12-15 =
+// pass-2 epilogue.
 #include <cuda.h>
 
 #include "kvc_internal.cuh"
@@ -52,7 +56,6 @@ constexpr int kFastThreads = 512;
 constexpr int kRows = 128;            // query rows per unit handled by one MMA (R <= 128)
 constexpr int kRunTiles = KVC_SCORE_RUN_TILES;
 constexpr int kGroupRuns = 8;         // runs whose partials are folded together at the first level
-constexpr int kJobSlots = 8;          // fold jobs that may wait in the CTA's queue
 constexpr int kQSlots = 3;
 constexpr int kPrefetch = KVC_SCORE_PREFETCH;
 constexpr float kLog2eF = 1.4426950408889634f;
@@ -64,8 +67,8 @@ constexpr int kMaxFastLayers = 112;   // 2 tensor maps per layer must fit the 32
 struct FastParams {
   CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (d, N, Hkv, Bt), box 64 x 128 x 1 x 1, 128-byte swizzle
   CUtensorMap q_maps[kMaxFastLayers];   // Q^(l) as (d, w, Hq, Bt), box 64 x w x G x 1
-  float4* partial;             // [U][RPU][32 lanes][2]: (ref, sum) of rows 4i .. 4i+3 of one run
-  float4* group_partial;       // [U][NG][32 lanes][2]: the same, folded over a group of runs
+  float4* partial;             // [U][RPU][64]: (ref, sum) of rows 2i and 2i+1 of one run
+  float4* group_partial;       // [U][NG][64]: the same, folded over a group of runs
   int* group_counter;          // [U][NG], preset to -1
   int* unit_counter;           // [U], preset to -1
   unsigned int* lse2;          // [U][128] fp32 bits, preset to 0xffffffff ("not there yet")
@@ -74,8 +77,10 @@ struct FastParams {
   int L, Bt, Hkv, G, R;
   long long N, q_pos0;
   int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
+  int step_u, step_j;          // grid = step_u * RPU + step_j: how a CTA's next run moves (unit, run in unit)
+  int step_l, step_b, step_h;  // step_u = (step_l * Bt + step_b) * Hkv + step_h
   unsigned int total_runs;     // U * RPU
-  long long shift;             // tiles by which the pass-2 stream trails the pass-1 stream
+  int shift;                   // tiles by which the pass-2 stream trails the pass-1 stream
   float sl2e;                  // scale * log2(e)
   int agg_group;
 };
@@ -158,7 +163,16 @@ __device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Wait for a TMEM load, tied to the registers it filled: the compiler may not use them before it.
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -204,6 +218,14 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const unsigned int* p) {
 __device__ __forceinline__ void st_relaxed_u32(unsigned int* p, uint32_t v) {
   asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_add_release(int* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_s32(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
   int old;
   asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
@@ -236,32 +258,48 @@ __device__ __forceinline__ void combine(float& M, float& Ls, float m, float l) {
 // The static per-CTA sequence.  Stream position idx -> (run ordinal, tile); a run is kRunTiles
 // consecutive tiles of one unit, runs are dealt to the CTAs round-robin.
 // ------------------------------------------------------------------------------------------------
-struct TileRef {
-  bool valid;
-  int t;        // position inside the run
-  int u;        // unit = (layer, sequence, KV head)
-  int j;        // run inside the unit
-  int tile;     // tile inside the unit
-  bool last;    // last valid tile of its run
+// Walks one stream of this CTA: position -> (run, tile).  Run k of the CTA is the global run
+// blockIdx.x + k * grid; the cursor moves from run to run by additions only (the per-run
+// increments come from the host), because a division would queue behind the exponentials in the
+// special-function pipe.
+struct Cursor {
+  int t;            // position inside the run, 0 .. kRunTiles-1
+  int u, j;         // unit, run inside the unit
+  int l, b, h;      // the unit's layer, sequence, KV head
+  __device__ __forceinline__ void init(const FastParams& P) {
+    t = 0;
+    u = (int)(blockIdx.x / (unsigned int)P.RPU);
+    j = (int)(blockIdx.x - (unsigned int)u * (unsigned int)P.RPU);
+    const int lb = u / P.Hkv;
+    h = u - lb * P.Hkv;
+    l = lb / P.Bt;
+    b = lb - l * P.Bt;
+  }
+  __device__ __forceinline__ int tile() const { return j * kRunTiles + t; }
+  __device__ __forceinline__ bool valid(const FastParams& P) const { return tile() < P.NT; }
+  // last valid tile of its run
+  __device__ __forceinline__ bool last(const FastParams& P) const { return t == kRunTiles - 1 || tile() + 1 >= P.NT; }
+  __device__ __forceinline__ void next_run(const FastParams& P) {
+    j += P.step_j;
+    int c = 0;
+    if (j >= P.RPU) { j -= P.RPU; c = 1; }
+    u += P.step_u + c;
+    h += P.step_h + c; c = 0;
+    if (h >= P.Hkv) { h -= P.Hkv; c = 1; }
+    b += P.step_b + c; c = 0;
+    if (b >= P.Bt) { b -= P.Bt; c = 1; }
+    l += P.step_l + c;
+  }
+  __device__ __forceinline__ void advance(const FastParams& P) {
+    if (++t == kRunTiles) { t = 0; next_run(P); }
+  }
 };
-__device__ __forceinline__ TileRef decode(const FastParams& P, long long idx) {
-  TileRef r;
-  const unsigned int k = (unsigned int)idx / kRunTiles;      // the host keeps every index below 2^31
-  r.t = (int)((unsigned int)idx - k * kRunTiles);
-  const unsigned int run = blockIdx.x + k * (unsigned int)P.grid;
-  r.u = (int)(run / (unsigned int)P.RPU);
-  r.j = (int)(run - (unsigned int)r.u * (unsigned int)P.RPU);
-  r.tile = r.j * kRunTiles + r.t;
-  r.valid = r.tile < P.NT;
-  r.last = r.valid && (r.t == kRunTiles - 1 || r.tile + 1 >= P.NT);
-  return r;
-}
-__device__ __forceinline__ void unit_coords(const FastParams& P, int u, int* l, int* b, int* h) {
-  const unsigned int lb = (unsigned int)u / (unsigned int)P.Hkv;
-  *h = (int)((unsigned int)u - lb * (unsigned int)P.Hkv);
-  *l = (int)(lb / (unsigned int)P.Bt);
-  *b = (int)(lb - (unsigned int)*l * (unsigned int)P.Bt);
-}
+
+// A ring position with its mbarrier phase bit.
+struct Ring {
+  int i, phase;
+  __device__ __forceinline__ void next(int n) { if (++i == n) { i = 0; phase ^= 1; } }
+};
 
 template <int D>
 struct SmemLayout {
@@ -277,16 +315,13 @@ struct SmemLayout {
   static constexpr int kBarTEmpty = kBarTFull + 32;
   static constexpr int kBarQFull = kBarTEmpty + 32;            // kQSlots x 8
   static constexpr int kBarQFree = kBarQFull + 8 * kQSlots;
-  static constexpr int kBarSFull = kBarQFree + 8 * kQSlots;    // statistics stage: full / empty
-  static constexpr int kBarSEmpty = kBarSFull + 8;
-  static constexpr int kTmemSlot = kBarSEmpty + 8;             // 4 B (+ padding)
+  static constexpr int kTmemSlot = kBarQFree + 8 * kQSlots;    // 4 B (+ padding)
   static constexpr int kAbort = kTmemSlot + 8;                 // 4 B
-  static constexpr int kJobHead = kAbort + 8;                  // 4 B: fold jobs pushed
-  static constexpr int kJobTail = kJobHead + 4;                // 4 B: fold jobs taken
-  static constexpr int kJobs = kJobTail + 4;                   // kJobSlots x 4 B
-  static constexpr int kNegLse = (kJobs + 4 * kJobSlots + 15) / 16 * 16;  // 128 floats, read as 16-byte vectors: -log-sum-exp of the pass-2 unit
-  static constexpr int kStats = kNegLse + kRows * 4;           // 2 halves x 128 rows x float2
-  static constexpr int kTotal = kStats + 2 * kRows * 8;
+  static constexpr int kFlushed = kAbort + 8;                  // 4 B: warps that have written a run's record
+  static constexpr int kNegLse = (kFlushed + 8 + 15) / 16 * 16;  // 128 floats, read as 16-byte vectors:
+                                                               // -log-sum-exp of the pass-2 unit
+  static constexpr int kStats = kNegLse + kRows * 4;           // 128 rows x float2: the upper half's statistics
+  static constexpr int kTotal = kStats + kRows * 8;
   static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
 
@@ -314,17 +349,13 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   auto bar_tempty = [&](int b) { return sbase + SL::kBarTEmpty + 8 * b; };
   auto bar_qfull = [&](int q) { return sbase + SL::kBarQFull + 8 * q; };
   auto bar_qfree = [&](int q) { return sbase + SL::kBarQFree + 8 * q; };
-  const uint32_t bar_sfull = sbase + SL::kBarSFull, bar_sempty = sbase + SL::kBarSEmpty;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < SL::kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
+    for (int s = 0; s < SL::kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 2); }
     for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), b < 2 ? 8 : 4); }
-    for (int q = 0; q < kQSlots; ++q) { mbar_init(bar_qfull(q), 1); mbar_init(bar_qfree(q), 1); }
-    mbar_init(bar_sfull, 8);
-    mbar_init(bar_sempty, 1);
+    for (int q = 0; q < kQSlots; ++q) { mbar_init(bar_qfull(q), 1); mbar_init(bar_qfree(q), 2); }
     *abort_word = 0;
-    *reinterpret_cast<volatile int*>(smem + SL::kJobHead) = 0;
-    *reinterpret_cast<volatile int*>(smem + SL::kJobTail) = 0;
+    *reinterpret_cast<volatile int*>(smem + SL::kFlushed) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -338,9 +369,10 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   const uint32_t tmem_base = *tmem_slot;
 
   // this CTA's share of the runs and the length of its sequence
-  const long long my_runs = (P.total_runs > blockIdx.x) ? (P.total_runs - blockIdx.x + P.grid - 1) / P.grid : 0;
-  const long long my_tiles = my_runs * kRunTiles;            // stream length (some positions hold no tile)
-  const long long n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
+  // (the host keeps all of these below 2^31)
+  const int my_runs = (P.total_runs > blockIdx.x) ? (int)((P.total_runs - blockIdx.x + P.grid - 1) / P.grid) : 0;
+  const int my_tiles = my_runs * kRunTiles;                  // stream length (some positions hold no tile)
+  const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
   const uint32_t q_bytes = (uint32_t)P.R * D * 2;
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
@@ -350,221 +382,208 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       unsigned long long pol_stream, pol_keep;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-      long long nk = 0;                // K tiles issued
-      long long qc = 0;                // Q tiles issued
+      Ring kr = {0, 0}, qr = {0, 0};   // next K stage / Q slot to fill; phase = parity of the fill count / ring size
+      int nk = 0, qc = 0;              // K tiles / Q tiles issued (saturating small counts are all that is needed)
       bool ok = true;
-      auto prefetch = [&](long long idx) {
-        if (idx >= my_tiles) return;
-        const TileRef t = decode(P, idx);
-        if (!t.valid) return;
-        int l, b, h;
-        unit_coords(P, t.u, &l, &b, &h);
-        for (int hf = 0; hf < SL::kHalves; ++hf) tma_prefetch_4d(P.k_maps + l, hf * 64, t.tile * kTile, h, b);
-      };
-      for (int i = 0; i < kPrefetch; ++i) prefetch(i);
-      for (long long i = 0; i < n_steps && ok; ++i) {
-        for (int pass = 0; pass < 2 && ok; ++pass) {
-          const long long idx = pass == 0 ? i : i - P.shift;
-          if (idx < 0 || idx >= my_tiles) continue;
-          const TileRef t = decode(P, idx);
-          if (!t.valid) continue;
-          int l, b, h;
-          unit_coords(P, t.u, &l, &b, &h);
-          if (t.t == 0) {                                    // a new run: its Q goes into the next ring slot
-            const int slot = (int)(qc % kQSlots);
-            if (qc >= kQSlots) {
-              ok = mbar_wait(bar_qfree(slot), (uint32_t)(((qc / kQSlots) - 1) & 1), abort_word);
-              if (!ok) break;
-            }
-            mbar_expect_tx(bar_qfull(slot), q_bytes);
-            for (int hf = 0; hf < SL::kHalves; ++hf)
-              tma_load_4d(sbase + SL::kQ + slot * SL::kTileBytes + hf * (kTile * 128), P.q_maps + l,
-                          bar_qfull(slot), hf * 64, 0, h * P.G, b, pol_keep);
-            ++qc;
-          }
-          const int s = (int)(nk % SL::kStages);
-          if (nk >= SL::kStages) {
-            ok = mbar_wait(bar_kempty(s), (uint32_t)(((nk / SL::kStages) - 1) & 1), abort_word);
-            if (!ok) break;
-          }
-          mbar_expect_tx(bar_kfull(s), SL::kTileBytes);
-          // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
+      Cursor cur[2], ahead;            // the two streams, and the pass-1 stream kPrefetch tiles ahead
+      cur[0].init(P); cur[1].init(P); ahead.init(P);
+      int ahead_pos = 0;
+      auto prefetch_next = [&]() {
+        if (ahead_pos >= my_tiles) return;
+        if (ahead.valid(P)) {
           for (int hf = 0; hf < SL::kHalves; ++hf)
-            tma_load_4d(sbase + SL::kK + s * SL::kTileBytes + hf * (kTile * 128), P.k_maps + l, bar_kfull(s),
-                        hf * 64, t.tile * kTile, h, b, pass == 0 ? pol_keep : pol_stream);
-          ++nk;
-          if (pass == 0) prefetch(idx + kPrefetch);
+            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile() * kTile, ahead.h, ahead.b);
         }
-      }
-      // drain: every issued copy must have landed before the CTA's shared memory is released
-      const long long first = nk > SL::kStages ? nk - SL::kStages : 0;
-      for (long long n = first; n < nk; ++n)
-        mbar_wait(bar_kfull((int)(n % SL::kStages)), (uint32_t)((n / SL::kStages) & 1), abort_word);
-      const long long qfirst = qc > kQSlots ? qc - kQSlots : 0;
-      for (long long n = qfirst; n < qc; ++n)
-        mbar_wait(bar_qfull((int)(n % kQSlots)), (uint32_t)((n / kQSlots) & 1), abort_word);
-    }
-  } else if (warp == 1) {
-    // ============================== MMA issuer =================================================
-    if (lane == 0) {
-      long long nk = 0, qc = 0;
-      long long nt[2] = {0, 0};        // tiles issued per pass
-      int cur_slot[2] = {0, 0};
-      bool ok = true;
-      for (long long i = 0; i < n_steps && ok; ++i) {
-        for (int pass = 0; pass < 2 && ok; ++pass) {
-          const long long idx = pass == 0 ? i : i - P.shift;
-          if (idx < 0 || idx >= my_tiles) continue;
-          const TileRef t = decode(P, idx);
-          if (!t.valid) continue;
-          if (t.t == 0) {
-            const int slot = (int)(qc % kQSlots);
-            ok = mbar_wait(bar_qfull(slot), (uint32_t)((qc / kQSlots) & 1), abort_word);
-            if (!ok) break;
-            cur_slot[pass] = slot;
-            ++qc;
-          }
-          const int s = (int)(nk % SL::kStages);
-          const int buf = pass * 2 + (int)(nt[pass] & 1);
-          ok = mbar_wait(bar_kfull(s), (uint32_t)((nk / SL::kStages) & 1), abort_word);
-          if (ok && nt[pass] >= 2)
-            ok = mbar_wait(bar_tempty(buf), (uint32_t)(((nt[pass] >> 1) - 1) & 1), abort_word);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t q_addr = sbase + SL::kQ + cur_slot[pass] * SL::kTileBytes;
-          const uint32_t k_addr = sbase + SL::kK + s * SL::kTileBytes;
-          const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (uint32_t)(kk >> 2) * (kTile * 128) + (uint32_t)(kk & 3) * 32;
-            const uint64_t dq = umma_desc(q_addr + off), dk = umma_desc(k_addr + off);
-            // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
-            if (pass == 0) tc_mma_bf16(d_tmem, dq, dk, kIdesc, kk > 0);
-            else tc_mma_bf16(d_tmem, dk, dq, kIdesc, kk > 0);
-          }
-          tc_commit(bar_kempty(s));      // the K stage may be refilled once these MMAs are done
-          tc_commit(bar_tfull(buf));     // ... and the accumulator is then complete
-          if (t.last) tc_commit(bar_qfree(cur_slot[pass]));
-          ++nk; ++nt[pass];
-        }
-      }
-    }
-  } else if (warp < 4) {
-    // ============================== statistics exchange ========================================
-    // Lane i owns rows 4i .. 4i+3.  A (reference, sum) record of 128 rows is 32 lanes x 2 float4.
-    volatile int* job_head = reinterpret_cast<volatile int*>(smem + SL::kJobHead);
-    volatile int* job_tail = reinterpret_cast<volatile int*>(smem + SL::kJobTail);
-    volatile int* jobs = reinterpret_cast<volatile int*>(smem + SL::kJobs);
-    if (warp == 2) {
-      // ---- push: one record per run, counted into its group; a completed group becomes a fold job
-      const float4* stage4 = reinterpret_cast<const float4*>(smem + SL::kStats);   // two rows per float4
-      int head = 0;
-      bool ok = true;
-      auto push_job = [&](int job) {                          // lane 0 only
-        const unsigned long long t0 = globaltimer_ns();
-        while (ok && head - *job_tail >= kJobSlots) {
-          __nanosleep(64);
-          if (*abort_word) ok = false;
-          else if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; ok = false; }
-        }
-        jobs[head % kJobSlots] = job;
-        __threadfence_block();
-        *job_head = ++head;
+        ahead.advance(P);
+        ++ahead_pos;
       };
-      for (long long k = 0; k < my_runs; ++k) {
-        const unsigned int run = blockIdx.x + (unsigned int)k * (unsigned int)P.grid;
-        const int u = (int)(run / (unsigned int)P.RPU);
-        const int j = (int)(run - (unsigned int)u * (unsigned int)P.RPU);
-        if (ok) ok = mbar_wait(bar_sfull, (uint32_t)(k & 1), abort_word);
-        float4 lo, hi;
-        {
-          const float4 a0 = stage4[2 * lane], a1 = stage4[2 * lane + 1];                       // tokens 0..63
-          const float4 b0 = stage4[kRows / 2 + 2 * lane], b1 = stage4[kRows / 2 + 2 * lane + 1];   // tokens 64..127
-          lo = a0; hi = a1;
-          combine(lo.x, lo.y, b0.x, b0.y);
-          combine(lo.z, lo.w, b0.z, b0.w);
-          combine(hi.x, hi.y, b1.x, b1.y);
-          combine(hi.z, hi.w, b1.z, b1.w);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_sempty);               // the stage may be overwritten
-        float4* dst = P.partial + (((long long)u * P.RPU + j) * 32 + lane) * 2;
-        dst[0] = lo;
-        dst[1] = hi;
-        __syncwarp();
-        if (lane == 0 && ok) {
-          const int g = j / kGroupRuns;
-          const int members = min(kGroupRuns, P.RPU - g * kGroupRuns);
-          const int old = atom_add_acq_rel(P.group_counter + (long long)u * P.NG + g, 1);
-          if (old == members - 2) push_job(u * P.NG + g);     // the counter starts at -1
-        }
-      }
-      if (lane == 0) push_job(-1);                            // no more jobs
-    } else {
-      // ---- fold: a group's records into one, and the last group of a unit into the log-sum-exp
-      int tail = 0;                                           // kept by lane 0
-      for (;;) {
-        int job = 0;
-        if (lane == 0) {
-          const unsigned long long t0 = globaltimer_ns();
-          while (*job_head == tail) {
-            __nanosleep(128);
-            if (*abort_word) { job = -1; break; }
-            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; job = -1; break; }
-          }
-          if (job == 0) {
-            job = jobs[tail % kJobSlots];
-            *job_tail = ++tail;
-          }
-        }
-        job = __shfl_sync(0xffffffffu, job, 0);
-        if (job < 0) break;
-        __threadfence();                                      // the records were published before the counts we saw
-        const int u = job / P.NG, g = job - u * P.NG;
-        const int members = min(kGroupRuns, P.RPU - g * kGroupRuns);
-        float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
-        {
-          const float4* src = P.partial + (((long long)u * P.RPU + g * kGroupRuns) * 32 + lane) * 2;
-          float4 v[2 * kGroupRuns];
+      for (int i = 0; i < kPrefetch; ++i) prefetch_next();
+      for (int i = 0; i < n_steps && ok; ++i) {
 #pragma unroll
-          for (int r = 0; r < kGroupRuns; ++r) {
-            if (r < members) { v[2 * r] = __ldcg(src + r * 64); v[2 * r + 1] = __ldcg(src + r * 64 + 1); }
-          }
-#pragma unroll
-          for (int r = 0; r < kGroupRuns; ++r) {
-            if (r < members) {
-              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
-              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
-              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
-              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
+        for (int pass = 0; pass < 2; ++pass) {
+          const int idx = pass == 0 ? i : i - P.shift;
+          if (!ok || idx < 0 || idx >= my_tiles) continue;
+          Cursor& c = cur[pass];
+          if (c.valid(P)) {
+            if (c.t == 0) {                                    // a new run: its Q goes into the next ring slot
+              if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), abort_word);
+              if (ok) {
+                mbar_expect_tx(bar_qfull(qr.i), q_bytes);
+                for (int hf = 0; hf < SL::kHalves; ++hf)
+                  tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
+                              bar_qfull(qr.i), hf * 64, 0, c.h * P.G, c.b, pol_keep);
+                qr.next(kQSlots);
+                if (qc < kQSlots) ++qc;
+              }
+            }
+            if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), abort_word);
+            if (ok) {
+              mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
+              // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
+              for (int hf = 0; hf < SL::kHalves; ++hf)
+                tma_load_4d(sbase + SL::kK + kr.i * SL::kTileBytes + hf * (kTile * 128), P.k_maps + c.l,
+                            bar_kfull(kr.i), hf * 64, c.tile() * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
+              kr.next(SL::kStages);
+              if (nk < SL::kStages) ++nk;
             }
           }
+          c.advance(P);
+          if (pass == 0) prefetch_next();
         }
-        float4* dst = P.group_partial + ((long long)job * 32 + lane) * 2;
+      }
+      // drain: every issued copy must have landed before the CTA's shared memory is released.
+      // The last fill of stage i is complete once its full barrier has left the phase of that fill.
+      for (int n = 0; n < nk; ++n) {
+        // walk the ring backwards from the slot before kr
+        int i2 = kr.i - 1 - n, ph = kr.phase;
+        if (i2 < 0) { i2 += SL::kStages; ph ^= 1; }
+        mbar_wait(bar_kfull(i2), (uint32_t)ph, abort_word);
+      }
+      for (int n = 0; n < qc; ++n) {
+        int i2 = qr.i - 1 - n, ph = qr.phase;
+        if (i2 < 0) { i2 += kQSlots; ph ^= 1; }
+        mbar_wait(bar_qfull(i2), (uint32_t)ph, abort_word);
+      }
+    }
+  } else if (warp < 3) {
+    // ============================== MMA issuers ================================================
+    // Both walk the whole sequence (the rings are shared and filled in sequence order) and each
+    // issues the tiles of its own pass.  Each also waits for the fills that belong to the other
+    // pass and acknowledges them: a parity wait is only meaningful for the phase that follows the
+    // last one seen, so neither thread may skip a phase of a ring barrier, and the producer must
+    // not refill a slot before both have seen its fill (the "empty" barriers count two arrivals:
+    // the user's commit and the other thread's acknowledgement).
+    if (lane == 0) {
+      const int mine = warp - 1;       // the pass this thread issues
+      Ring kr = {0, 0}, qr = {0, 0};
+      Ring tb = {0, 0};                // accumulator buffer of this pass (two per pass)
+      int nt = 0;                      // tiles issued (saturating at 2)
+      int cur_slot = 0;
+      bool ok = true;
+      Cursor cur[2];
+      cur[0].init(P); cur[1].init(P);
+      for (int i = 0; i < n_steps && ok; ++i) {
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+          const int idx = pass == 0 ? i : i - P.shift;
+          if (!ok || idx < 0 || idx >= my_tiles) continue;
+          Cursor& c = cur[pass];
+          if (c.valid(P)) {
+            if (c.t == 0) {
+              ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, abort_word);
+              if (pass == mine) cur_slot = qr.i;
+              else if (ok) mbar_arrive(bar_qfree(qr.i));
+            }
+            if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word);
+            if (ok && pass != mine) mbar_arrive(bar_kempty(kr.i));
+            if (pass == mine) {
+              const int buf = pass * 2 + tb.i;
+              if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), abort_word);
+              if (ok) {
+                tc_fence_after();
+                const uint64_t dq0 = umma_desc(sbase + SL::kQ + cur_slot * SL::kTileBytes);
+                const uint64_t dk0 = umma_desc(sbase + SL::kK + kr.i * SL::kTileBytes);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                  // the start-address field counts 16-byte units: 64-element half, then 32 B per K step
+                  const uint64_t off = (uint64_t)(((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4);
+                  // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
+                  if (pass == 0) tc_mma_bf16(d_tmem, dq0 + off, dk0 + off, kIdesc, kk > 0);
+                  else tc_mma_bf16(d_tmem, dk0 + off, dq0 + off, kIdesc, kk > 0);
+                }
+                tc_commit(bar_kempty(kr.i));   // the K stage may be refilled once these MMAs are done
+                tc_commit(bar_tfull(buf));     // ... and the accumulator is then complete
+                if (c.last(P)) tc_commit(bar_qfree(cur_slot));
+                tb.next(2);
+                if (nt < 2) ++nt;
+              }
+            }
+            if (c.t == 0) qr.next(kQSlots);
+            kr.next(SL::kStages);
+          }
+          c.advance(P);
+        }
+      }
+    }
+  } else if (warp == 3) {
+    // ============================== statistics exchange ========================================
+    // This CTA folds the groups  x, x + grid, ...  (x = blockIdx.x; a group is numbered
+    // unit * NG + group) and the units  x, x + grid, ...   Jobs are taken in the order in which
+    // they become ready anywhere in the grid -- a group before every unit whose last group is
+    // not smaller -- so a wait here only ever depends on jobs that are earlier in that order.
+    // Lane i owns rows 4i .. 4i+3; a record of 128 rows is 64 float4, two per lane.
+    const int n_groups = P.U * P.NG;
+    int gi = blockIdx.x, un = blockIdx.x;             // next group / next unit of this CTA
+    bool ok = true;
+    while (ok && (gi < n_groups || un < P.U)) {
+      const bool take_group = gi < n_groups && (un >= P.U || gi <= (un + 1) * P.NG - 1);
+      const int* counter = take_group ? P.group_counter + gi : P.unit_counter + un;
+      int target;                                     // the counters start at -1
+      if (take_group) {
+        const int g = gi % P.NG;
+        target = min(kGroupRuns, P.RPU - g * kGroupRuns) - 1;
+      } else {
+        target = P.NG - 1;
+      }
+      if (lane == 0) {
+        const unsigned long long t0 = globaltimer_ns();
+        uint32_t spins = 0;
+        while (ld_acquire_s32(counter) != target) {
+          __nanosleep(200);
+          if ((++spins & 63u) == 0) {
+            if (*abort_word) { ok = false; break; }
+            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; ok = false; break; }
+          }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      __threadfence();                                // the records were published before the counts we saw
+      float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
+      if (take_group) {
+        const int u = gi / P.NG, g = gi - u * P.NG;
+        const int members = target + 1;
+        const float4* src = P.partial + ((long long)u * P.RPU + g * kGroupRuns) * 64 + 2 * lane;
+        float4 v[2 * kGroupRuns];
+#pragma unroll
+        for (int r = 0; r < kGroupRuns; ++r) {
+          if (r < members) { v[2 * r] = __ldcg(src + r * 64); v[2 * r + 1] = __ldcg(src + r * 64 + 1); }
+        }
+#pragma unroll
+        for (int r = 0; r < kGroupRuns; ++r) {
+          if (r < members) {
+            combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
+            combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
+            combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
+            combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
+          }
+        }
+        float4* dst = P.group_partial + (long long)gi * 64 + 2 * lane;
         dst[0] = lo;
         dst[1] = hi;
         __syncwarp();
-        int last = 0;
-        if (lane == 0) last = (atom_add_acq_rel(P.unit_counter + u, 1) == P.NG - 2) ? 1 : 0;
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
+        if (lane == 0) {
           __threadfence();
-          const float4* src = P.group_partial + ((long long)u * P.NG * 32 + lane) * 2;
-          lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f); hi = lo;
-#pragma unroll 4
-          for (int r = 0; r < P.NG; ++r) {
-            const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
-            combine(lo.x, lo.y, v0.x, v0.y);
-            combine(lo.z, lo.w, v0.z, v0.w);
-            combine(hi.x, hi.y, v1.x, v1.y);
-            combine(hi.z, hi.w, v1.z, v1.w);
-          }
-          unsigned int* out = P.lse2 + (long long)u * kRows + 4 * lane;
-          st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
-          st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
-          st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
-          st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
+          red_add_release(P.unit_counter + u, 1);
         }
+        gi += P.grid;
+      } else {
+        const float4* src = P.group_partial + (long long)un * P.NG * 64 + 2 * lane;
+#pragma unroll 4
+        for (int r = 0; r < P.NG; ++r) {
+          const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
+          combine(lo.x, lo.y, v0.x, v0.y);
+          combine(lo.z, lo.w, v0.z, v0.w);
+          combine(hi.x, hi.y, v1.x, v1.y);
+          combine(hi.z, hi.w, v1.z, v1.w);
+        }
+        unsigned int* out = P.lse2 + (long long)un * kRows + 4 * lane;
+        st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
+        st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
+        st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
+        st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
+        un += P.grid;
       }
     }
   } else if (warp < 12) {
@@ -574,11 +593,11 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const int row = quarter * 32 + lane;              // TMEM lane = query row
     const bool row_used = row < P.R;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + half * kRows + row;
+    float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + row;
     const long long row_vis = min(P.N - 1, P.q_pos0 + (row % W));     // last key this row sees
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
 
-    long long n1 = 0, runs_done = 0;
+    int n1 = 0;
     float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
     bool ok = true;
 
@@ -630,18 +649,22 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       else slow_chunk(r, c_first, false);               // a logit far above the reference: move it
     };
 
-    for (long long idx = 0; idx < my_tiles; ++idx) {
-      const TileRef t = decode(P, idx);
-      if (!t.valid) continue;
-      const int buf = (int)(n1 & 1);
+    Cursor c;
+    c.init(P);
+    for (int idx = 0; idx < my_tiles; ++idx, c.advance(P)) {
+      if (!c.valid(P)) continue;
+      const int tile = c.tile();
+      const bool run_ends = c.last(P);
+      const int buf = n1 & 1;
       if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word);
       tc_fence_after();
-      const long long c0 = (long long)t.tile * kTile + half * 64;
-      const bool full = (long long)t.tile * kTile + kTile - 1 <= vis_all;     // no masking anywhere in the tile
+      const long long c0 = (long long)tile * kTile + half * 64;
+      const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;       // no masking anywhere in the tile
       uint32_t ra[32], rb[32];
       tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64, ra);
       tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64 + 32, rb);
-      tc_wait_ld();
+      tc_wait_ld(ra);
+      tc_wait_ld(rb);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty(buf));      // the accumulator is in registers now
@@ -655,13 +678,27 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           slow_chunk(rb, c0 + 32, true);
         }
       }
-      if (t.last) {
-        // hand the run's (reference, sum) to the exchange warps
-        if (ok && runs_done >= 1) ok = mbar_wait(bar_sempty, (uint32_t)((runs_done - 1) & 1), abort_word);
-        *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_sfull);
-        ++runs_done;
+      if (run_ends) {
+        // the two halves of every row meet through shared memory; the lower half's warps write
+        // the run's record and report it to the statistics warp
+        if (half == 1) *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
+        named_bar(3, 256);
+        const float2 other = *stage;
+        named_bar(3, 256);                             // the stage may be written again
+        if (half == 0) {
+          float M = row_used ? mref : -INFINITY, Ls = row_used ? lsum : 0.f;
+          combine(M, Ls, other.x, other.y);
+          reinterpret_cast<float2*>(P.partial)[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
+          __syncwarp();
+          if (lane == 0) {
+            __threadfence();                            // this warp's part of the record, device-wide
+            const int seen = atomicAdd(reinterpret_cast<int*>(smem + SL::kFlushed), 1);
+            if ((seen & 3) == 3) {                      // the other three warps' parts are out as well
+              __threadfence();
+              red_add_release(P.group_counter + (long long)c.u * P.NG + c.j / kGroupRuns, 1);
+            }
+          }
+        }
         mref = -INFINITY; lsum = 0.f;
       }
     }
@@ -673,17 +710,19 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     float* neg_lse = reinterpret_cast<float*>(smem + SL::kNegLse);
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
     const int n_chunks = (P.R + 31) / 32;
-    long long n2 = 0;
+    int n2 = 0;
     bool ok = true;
 
-    for (long long idx = 0; idx < my_tiles; ++idx) {
-      const TileRef t = decode(P, idx);
-      if (!t.valid) continue;
-      if (t.t == 0) {
+    Cursor cu;
+    cu.init(P);
+    for (int idx = 0; idx < my_tiles; ++idx, cu.advance(P)) {
+      if (!cu.valid(P)) continue;
+      const int tile = cu.tile();
+      if (cu.t == 0) {
         // a new run: wait for its unit's log-sum-exp (the value itself is the flag)
         uint32_t bits = 0xffffffffu;
         if (ok && trow < P.R) {
-          const unsigned int* src = P.lse2 + (long long)t.u * kRows + trow;
+          const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
           bits = ld_relaxed_u32(src);
           if (bits == 0xffffffffu) {
             const unsigned long long t0 = globaltimer_ns();
@@ -702,67 +741,83 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         named_bar(1, 128);
         if (*abort_word) ok = false;
       }
-      const int buf = 2 + (int)(n2 & 1);
+      const int buf = 2 + (n2 & 1);
+      const uint32_t tmem_col = (uint32_t)buf * kTile;
       if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), abort_word);
+      ++n2;
       tc_fence_after();
-      const long long c = (long long)t.tile * kTile + trow;          // this thread's token
-      const bool full = (long long)t.tile * kTile + kTile - 1 <= vis_all;
+      const long long c = (long long)tile * kTile + trow;            // this thread's token
+      const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;
       const long long m_min = c - P.q_pos0;                           // rows m >= m_min see token c
       float gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
       float hacc = kTaskMean ? 0.f : -INFINITY;
+      float head_max[kRows / 32];                                     // fast path: log2 of S_task per query head
       uint32_t r[32];
-      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile, r);
-#pragma unroll 1
-      for (int j = 0; j < n_chunks; ++j) {
-        tc_wait_ld();
-        float x[32];
-        {
-          const ulonglong2* l2 = reinterpret_cast<const ulonglong2*>(neg_lse + j * 32);
+      tc_ld32_nowait(lane_addr + tmem_col, r);
+#pragma unroll
+      for (int j = 0; j < kRows / 32; ++j) {
+        if (j < n_chunks) {
+          // the rows' -log-sum-exp for this chunk, fetched while the accumulator load is in flight
+          ulonglong2 nl[8];
+          {
+            const ulonglong2* l2 = reinterpret_cast<const ulonglong2*>(neg_lse + j * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) nl[i] = l2[i];
+          }
+          tc_wait_ld(r);
+          float x[32];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const ulonglong2 nl = l2[i];
-            const unsigned long long y0 = fma2(pack2u(r[4 * i], r[4 * i + 1]), scale2, nl.x);
-            const unsigned long long y1 = fma2(pack2u(r[4 * i + 2], r[4 * i + 3]), scale2, nl.y);
+            const unsigned long long y0 = fma2(pack2u(r[4 * i], r[4 * i + 1]), scale2, nl[i].x);
+            const unsigned long long y1 = fma2(pack2u(r[4 * i + 2], r[4 * i + 3]), scale2, nl[i].y);
             unpack2(y0, x[4 * i], x[4 * i + 1]);                     // log2 of the attention weights
             unpack2(y1, x[4 * i + 2], x[4 * i + 3]);
           }
-        }
-        if (j + 1 < n_chunks) tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + (j + 1) * 32, r);
-        if (!kTaskMean && full && W >= 32) {
-          // the whole chunk belongs to one query head
-          float a = x[0], b = x[1];
-#pragma unroll
-          for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
-          hacc = max3(hacc, a, b);
-          hacc = max3(hacc, x[30], x[31]);
-          if (((j + 1) * 32) % W == 0) {
-            const float s_task = ex2(hacc);
-            gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
-            hacc = -INFINITY;
+          if (j + 1 < n_chunks) {
+            tc_ld32_nowait(lane_addr + tmem_col + (j + 1) * 32, r);
+          } else {
+            tc_fence_before();                                        // the accumulator has been read
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty(buf));
           }
-        } else {
+          if (!kTaskMean && full && W >= 32) {
+            // the whole chunk belongs to one query head
+            float a = x[0], b = x[1];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int col = j * 32 + i;
-            float xi = x[i];
-            if (!full && (col % W) < m_min) xi = -INFINITY;
-            if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
-            if ((col + 1) % W == 0) {                                  // a query head is complete
-              if (col < P.R) {
-                const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
-                gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+            for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
+            hacc = max3(hacc, a, b);
+            hacc = max3(hacc, x[30], x[31]);
+            if (((j + 1) * 32) % W == 0) { head_max[j] = hacc; hacc = -INFINITY; }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int col = j * 32 + i;
+              float xi = x[i];
+              if (!full && (col % W) < m_min) xi = -INFINITY;
+              if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
+              if ((col + 1) % W == 0) {                                // a query head is complete
+                if (col < P.R) {
+                  const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
+                  gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+                }
+                hacc = kTaskMean ? 0.f : -INFINITY;
               }
-              hacc = kTaskMean ? 0.f : -INFINITY;
             }
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty(buf));
-      ++n2;
+      if (!kTaskMean && full && W >= 32) {
+        // the exponentials of all heads together, off the per-chunk path
+#pragma unroll
+        for (int j = 0; j < kRows / 32; ++j) {
+          if (j < n_chunks && ((j + 1) * 32) % W == 0) {
+            const float s_task = ex2(head_max[j]);
+            gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+          }
+        }
+      }
       if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
-      if (ok && c < P.N) P.scores[(long long)t.u * P.N + c] = gacc;
+      if (ok && c < P.N) P.scores[(long long)cu.u * P.N + c] = gacc;
     }
   }
 
@@ -924,7 +979,11 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G; fp.R = G * P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
   fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.NG = pl.NG; fp.grid = pl.grid;
-  fp.total_runs = (unsigned int)pl.total_runs; fp.shift = pl.shift;
+  fp.total_runs = (unsigned int)pl.total_runs; fp.shift = (int)pl.shift;
+  fp.step_u = pl.grid / pl.RPU; fp.step_j = pl.grid % pl.RPU;
+  fp.step_h = fp.step_u % P.Hkv;
+  fp.step_b = (fp.step_u / P.Hkv) % P.Bt;
+  fp.step_l = fp.step_u / P.Hkv / P.Bt;
   fp.sl2e = P.scale * kLog2eF;
   fp.agg_group = P.agg_group;
   const bool mean = P.agg_task == KVC_AGG_MEAN;
