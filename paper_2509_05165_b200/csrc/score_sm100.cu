@@ -31,9 +31,9 @@
 // Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch); warp 1 = MMA
 // issuer of pass 1 and TMEM owner; warp 2 = MMA issuer of pass 2 (two issuers, because the
 // waits, commits and bookkeeping around a tile cost one thread more time than the tile's MMAs
-// take, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-11 =
-// pass-1 epilogue (two warpgroups, each takes one half of every tile's columns); warps 12-15 =
-// pass-2 epilogue.
+// take, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-7 =
+// pass-2 epilogue; warps 8-15 = pass-1 epilogue (two warpgroups, each takes one half of every
+// tile's columns).
 #include <cuda.h>
 
 #include "kvc_internal.cuh"
@@ -115,8 +115,9 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the abort word is set or the time limit expires (and sets it).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word) {
-  if (mbar_try(bar, parity)) return true;
+// The retry loop is kept out of line: the kernel's hot loops have to stay small enough for the
+// instruction cache, which sixteen warps in six different roles share.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
   while (!mbar_try(bar, parity)) {
@@ -126,6 +127,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
   return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_word);
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3, unsigned long long policy) {
@@ -324,6 +329,78 @@ struct SmemLayout {
   static constexpr int kTotal = kStats + kRows * 8;
   static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
+
+// ------------------------------------------------------------------------------------------------
+// Cold paths, out of line: tiles that touch the causal boundary or the end of the context, and
+// the aggregator variants other than the paper's defaults.
+// ------------------------------------------------------------------------------------------------
+
+// Pass 1, 64 columns (tokens c_first ..) of this thread's query row, with masking: the row's
+// (reference, sum) follows the running maximum.  Reads the accumulator itself.
+__device__ __noinline__ void p1_masked_half(uint32_t taddr, long long c_first, long long row_vis, float sl2e,
+                                            float* mref_io, float* lsum_io) {
+  float mref = *mref_io, lsum = *lsum_io;
+#pragma unroll 1
+  for (int part = 0; part < 2; ++part) {
+    uint32_t r[32];
+    tc_ld32_nowait(taddr + part * 32, r);
+    tc_wait_ld(r);
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      v[i] = __uint_as_float(r[i]);
+      if (c_first + part * 32 + i > row_vis) v[i] = -INFINITY;
+    }
+    float x0 = v[0], x1 = v[1];
+#pragma unroll
+    for (int i = 2; i < 32; i += 2) { x0 = max3(x0, v[i], v[i + 1]); }
+    const float m_new = fmaxf(mref, fmaxf(x0, x1) * sl2e);
+    if (m_new > -INFINITY) {
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+      for (int i = 0; i < 32; i += 4) {
+        a0 += ex2(fmaf(v[i + 0], sl2e, -m_new));
+        a1 += ex2(fmaf(v[i + 1], sl2e, -m_new));
+        a2 += ex2(fmaf(v[i + 2], sl2e, -m_new));
+        a3 += ex2(fmaf(v[i + 3], sl2e, -m_new));
+      }
+      lsum = lsum * ex2(mref - m_new) + ((a0 + a1) + (a2 + a3));
+      mref = m_new;
+    }
+  }
+  *mref_io = mref;
+  *lsum_io = lsum;
+}
+
+// Pass 2, one token (this thread's TMEM lane) against all query rows, any aggregator, with
+// masking.  Returns the group aggregate before the division of the mean.
+template <int W, bool kTaskMean>
+__device__ __noinline__ float p2_generic_tile(uint32_t taddr, const float* neg_lse, int n_chunks, int R, float sl2e,
+                                              bool full, long long m_min, int agg_group) {
+  float gacc = (agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
+  float hacc = kTaskMean ? 0.f : -INFINITY;
+#pragma unroll 1
+  for (int j = 0; j < n_chunks; ++j) {
+    uint32_t r[32];
+    tc_ld32_nowait(taddr + j * 32, r);
+    tc_wait_ld(r);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int col = j * 32 + i;
+      float xi = fmaf(__uint_as_float(r[i]), sl2e, neg_lse[col]);       // log2 of the attention weight
+      if (!full && (col % W) < m_min) xi = -INFINITY;
+      if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
+      if ((col + 1) % W == 0) {                                          // a query head is complete
+        if (col < R) {
+          const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
+          gacc = (agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+        }
+        hacc = kTaskMean ? 0.f : -INFINITY;
+      }
+    }
+  }
+  return gacc;
+}
 
 // ------------------------------------------------------------------------------------------------
 // The kernel
@@ -586,9 +663,9 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         un += P.grid;
       }
     }
-  } else if (warp < 12) {
+  } else if (warp >= 8) {
     // ============================== pass-1 epilogue ============================================
-    const int half = (warp - 4) >> 2;                 // which 64 columns (tokens) of every tile
+    const int half = (warp - 8) >> 2;                 // which 64 columns (tokens) of every tile
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;              // TMEM lane = query row
     const bool row_used = row < P.R;
@@ -601,52 +678,33 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
     bool ok = true;
 
-    // 32 logits with masking and a reference that follows the maximum
-    auto slow_chunk = [&](const uint32_t (&r)[32], long long c_first, bool masked) {
-      float v[32];
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        v[i] = __uint_as_float(r[i]);
-        if (masked && c_first + i > row_vis) v[i] = -INFINITY;
-      }
-      float x0 = v[0], x1 = v[1];
-#pragma unroll
-      for (int i = 2; i < 32; i += 2) { x0 = max3(x0, v[i], v[i + 1]); }
-      const float m_new = fmaxf(mref, fmaxf(x0, x1) * P.sl2e);
-      if (m_new > -INFINITY) {
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    // 32 unmasked logits against the row's current reference: no maximum, packed arithmetic.
+    // Any logit of the row will do as a reference; if a chunk's sum leaves the range of fp32
+    // the reference is moved up by 64 and the chunk is summed again.
+    auto fast_chunk = [&](const uint32_t (&r)[32]) {
+      if (mref == -INFINITY) mref = __uint_as_float(r[0]) * P.sl2e;
+#pragma unroll 1
+      for (int attempt = 0; attempt < 8; ++attempt) {
+        const unsigned long long neg_ref = pack2(-mref, -mref);
+        unsigned long long acc0 = 0ull, acc1 = 0ull;      // +0.0f twice
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
-          a0 += ex2(fmaf(v[i + 0], P.sl2e, -m_new));
-          a1 += ex2(fmaf(v[i + 1], P.sl2e, -m_new));
-          a2 += ex2(fmaf(v[i + 2], P.sl2e, -m_new));
-          a3 += ex2(fmaf(v[i + 3], P.sl2e, -m_new));
+          const unsigned long long y0 = fma2(pack2u(r[i], r[i + 1]), scale2, neg_ref);
+          const unsigned long long y1 = fma2(pack2u(r[i + 2], r[i + 3]), scale2, neg_ref);
+          float a, b, c, d;
+          unpack2(y0, a, b);
+          unpack2(y1, c, d);
+          acc0 = add2(acc0, pack2(ex2(a), ex2(b)));
+          acc1 = add2(acc1, pack2(ex2(c), ex2(d)));
         }
-        lsum = lsum * ex2(mref - m_new) + ((a0 + a1) + (a2 + a3));
-        mref = m_new;
+        float s0, s1, s2, s3;
+        unpack2(acc0, s0, s1);
+        unpack2(acc1, s2, s3);
+        const float sum = (s0 + s1) + (s2 + s3);
+        if (sum < kRescaleLimit) { lsum += sum; break; }   // (false for inf / NaN as well)
+        mref += 64.f;
+        lsum *= 5.421010862427522e-20f;                    // 2^-64
       }
-    };
-    // 32 unmasked logits against the current reference: no maximum, packed arithmetic
-    auto fast_chunk = [&](const uint32_t (&r)[32], long long c_first) {
-      if (mref == -INFINITY) { slow_chunk(r, c_first, false); return; }
-      const unsigned long long neg_ref = pack2(-mref, -mref);
-      unsigned long long acc0 = 0ull, acc1 = 0ull;      // +0.0f twice
-#pragma unroll
-      for (int i = 0; i < 32; i += 4) {
-        const unsigned long long y0 = fma2(pack2u(r[i], r[i + 1]), scale2, neg_ref);
-        const unsigned long long y1 = fma2(pack2u(r[i + 2], r[i + 3]), scale2, neg_ref);
-        float a, b, c, d;
-        unpack2(y0, a, b);
-        unpack2(y1, c, d);
-        acc0 = add2(acc0, pack2(ex2(a), ex2(b)));
-        acc1 = add2(acc1, pack2(ex2(c), ex2(d)));
-      }
-      float s0, s1, s2, s3;
-      unpack2(acc0, s0, s1);
-      unpack2(acc1, s2, s3);
-      const float s = (s0 + s1) + (s2 + s3);
-      if (s < kRescaleLimit) lsum += s;                 // also false for inf / NaN
-      else slow_chunk(r, c_first, false);               // a logit far above the reference: move it
     };
 
     Cursor c;
@@ -660,23 +718,28 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       tc_fence_after();
       const long long c0 = (long long)tile * kTile + half * 64;
       const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;       // no masking anywhere in the tile
-      uint32_t ra[32], rb[32];
-      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64, ra);
-      tc_ld32_nowait(lane_addr + (uint32_t)buf * kTile + half * 64 + 32, rb);
-      tc_wait_ld(ra);
-      tc_wait_ld(rb);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty(buf));      // the accumulator is in registers now
+      const uint32_t taddr = lane_addr + (uint32_t)buf * kTile + half * 64;
       ++n1;
-      if (ok && row_used) {
-        if (full) {
-          fast_chunk(ra, c0);
-          fast_chunk(rb, c0 + 32);
-        } else {
-          slow_chunk(ra, c0, true);
-          slow_chunk(rb, c0 + 32, true);
+      if (full) {
+        uint32_t ra[32], rb[32];
+        tc_ld32_nowait(taddr, ra);
+        tc_ld32_nowait(taddr + 32, rb);
+        tc_wait_ld(ra);
+        tc_wait_ld(rb);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(buf));    // the accumulator is in registers now
+        if (ok && row_used) {
+          fast_chunk(ra);
+          fast_chunk(rb);
         }
+      } else {
+        float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
+        p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
+        if (ok && row_used) { mref = m2; lsum = l2; }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(buf));
       }
       if (run_ends) {
         // the two halves of every row meet through shared memory; the lower half's warps write
@@ -748,15 +811,16 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       tc_fence_after();
       const long long c = (long long)tile * kTile + trow;            // this thread's token
       const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;
-      const long long m_min = c - P.q_pos0;                           // rows m >= m_min see token c
-      float gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
-      float hacc = kTaskMean ? 0.f : -INFINITY;
-      float head_max[kRows / 32];                                     // fast path: log2 of S_task per query head
-      uint32_t r[32];
-      tc_ld32_nowait(lane_addr + tmem_col, r);
-#pragma unroll
-      for (int j = 0; j < kRows / 32; ++j) {
-        if (j < n_chunks) {
+      float gacc;
+      if (!kTaskMean && W >= 32 && full) {
+        // the paper's default (max over the window) on a tile no mask touches: every 32-column
+        // chunk belongs to one query head
+        gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
+        float hacc = -INFINITY;
+        uint32_t r[32];
+        tc_ld32_nowait(lane_addr + tmem_col, r);
+#pragma unroll 1
+        for (int j = 0; j < n_chunks; ++j) {
           // the rows' -log-sum-exp for this chunk, fetched while the accumulator load is in flight
           ulonglong2 nl[8];
           {
@@ -780,41 +844,23 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty(buf));
           }
-          if (!kTaskMean && full && W >= 32) {
-            // the whole chunk belongs to one query head
-            float a = x[0], b = x[1];
+          float a = x[0], b = x[1];
 #pragma unroll
-            for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
-            hacc = max3(hacc, a, b);
-            hacc = max3(hacc, x[30], x[31]);
-            if (((j + 1) * 32) % W == 0) { head_max[j] = hacc; hacc = -INFINITY; }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int col = j * 32 + i;
-              float xi = x[i];
-              if (!full && (col % W) < m_min) xi = -INFINITY;
-              if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
-              if ((col + 1) % W == 0) {                                // a query head is complete
-                if (col < P.R) {
-                  const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
-                  gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
-                }
-                hacc = kTaskMean ? 0.f : -INFINITY;
-              }
-            }
-          }
-        }
-      }
-      if (!kTaskMean && full && W >= 32) {
-        // the exponentials of all heads together, off the per-chunk path
-#pragma unroll
-        for (int j = 0; j < kRows / 32; ++j) {
-          if (j < n_chunks && ((j + 1) * 32) % W == 0) {
-            const float s_task = ex2(head_max[j]);
+          for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
+          hacc = max3(hacc, a, b);
+          hacc = max3(hacc, x[30], x[31]);
+          if (((j + 1) * 32) % W == 0) {
+            const float s_task = ex2(hacc);
             gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+            hacc = -INFINITY;
           }
         }
+      } else {
+        gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, P.R, P.sl2e, full,
+                                             c - P.q_pos0, P.agg_group);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(buf));
       }
       if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
       if (ok && c < P.N) P.scores[(long long)cu.u * P.N + c] = gacc;
