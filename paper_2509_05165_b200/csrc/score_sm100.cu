@@ -49,6 +49,21 @@
 #endif
 
 namespace kvc {
+#ifdef KVC_SCORE_TRACE
+// Optional trace (debug builds only): per CTA, SM clocks each role spent in each kind of wait.
+__device__ unsigned long long g_score_trace[160 * 24];
+#define KVC_TR_DECL(...) long long __VA_ARGS__
+#define KVC_TR(acc, stmt) do { const long long _t0 = clock64(); stmt; acc += clock64() - _t0; } while (0)
+#define KVC_TR_SINCE(acc, start) acc += clock64() - (start)
+#define KVC_TR_PUT(i, v) g_score_trace[blockIdx.x * 24 + (i)] = (unsigned long long)(v)
+#define KVC_TR_NOW() clock64()
+#else
+#define KVC_TR_SINCE(acc, start)
+#define KVC_TR_DECL(...)
+#define KVC_TR(acc, stmt) do { stmt; } while (0)
+#define KVC_TR_PUT(i, v)
+#define KVC_TR_NOW() 0ll
+#endif
 namespace {
 
 constexpr int kTile = 128;            // tokens per tile = MMA M = MMA N
@@ -231,9 +246,9 @@ __device__ __forceinline__ int ld_acquire_s32(const int* p) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+__device__ __forceinline__ int atom_add_acq_rel_cta_shared(uint32_t saddr, int v) {
   int old;
-  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  asm volatile("atom.acq_rel.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(saddr), "r"(v) : "memory");
   return old;
 }
 
@@ -329,6 +344,20 @@ struct SmemLayout {
   static constexpr int kTotal = kStats + kRows * 8;
   static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
+
+// Bounded poll of a log-sum-exp slot (the value itself is the flag).
+__device__ __noinline__ uint32_t poll_lse_slow(const unsigned int* src, volatile int* abort_word) {
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0, bits;
+  while ((bits = ld_relaxed_u32(src)) == 0xffffffffu) {
+    __nanosleep(100);
+    if ((++spins & 255u) == 0) {
+      if (*abort_word) break;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
+    }
+  }
+  return bits;
+}
 
 // ------------------------------------------------------------------------------------------------
 // Cold paths, out of line: tiles that touch the causal boundary or the end of the context, and
@@ -459,6 +488,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       unsigned long long pol_stream, pol_keep;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+      KVC_TR_DECL(w_q = 0, w_k = 0, w_s = KVC_TR_NOW());
       Ring kr = {0, 0}, qr = {0, 0};   // next K stage / Q slot to fill; phase = parity of the fill count / ring size
       int nk = 0, qc = 0;              // K tiles / Q tiles issued (saturating small counts are all that is needed)
       bool ok = true;
@@ -483,7 +513,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           Cursor& c = cur[pass];
           if (c.valid(P)) {
             if (c.t == 0) {                                    // a new run: its Q goes into the next ring slot
-              if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), abort_word);
+              KVC_TR(w_q, if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), abort_word));
               if (ok) {
                 mbar_expect_tx(bar_qfull(qr.i), q_bytes);
                 for (int hf = 0; hf < SL::kHalves; ++hf)
@@ -493,7 +523,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 if (qc < kQSlots) ++qc;
               }
             }
-            if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), abort_word);
+            KVC_TR(w_k, if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), abort_word));
             if (ok) {
               mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
               // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
@@ -508,6 +538,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           if (pass == 0) prefetch_next();
         }
       }
+      KVC_TR_PUT(0, w_q); KVC_TR_PUT(1, w_k); KVC_TR_PUT(2, KVC_TR_NOW() - w_s);
       // drain: every issued copy must have landed before the CTA's shared memory is released.
       // The last fill of stage i is complete once its full barrier has left the phase of that fill.
       for (int n = 0; n < nk; ++n) {
@@ -537,6 +568,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       int nt = 0;                      // tiles issued (saturating at 2)
       int cur_slot = 0;
       bool ok = true;
+      KVC_TR_DECL(m_q = 0, m_ko = 0, m_kx = 0, m_t = 0, m_i = 0, m_s = KVC_TR_NOW());
       Cursor cur[2];
       cur[0].init(P); cur[1].init(P);
       for (int i = 0; i < n_steps && ok; ++i) {
@@ -547,15 +579,17 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           Cursor& c = cur[pass];
           if (c.valid(P)) {
             if (c.t == 0) {
-              ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, abort_word);
+              KVC_TR(m_q, ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, abort_word));
               if (pass == mine) cur_slot = qr.i;
               else if (ok) mbar_arrive(bar_qfree(qr.i));
             }
-            if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word);
+            if (pass == mine) KVC_TR(m_ko, if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word));
+            else KVC_TR(m_kx, if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word));
             if (ok && pass != mine) mbar_arrive(bar_kempty(kr.i));
             if (pass == mine) {
               const int buf = pass * 2 + tb.i;
-              if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), abort_word);
+              KVC_TR(m_t, if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), abort_word));
+              KVC_TR_DECL(m_i0 = KVC_TR_NOW());
               if (ok) {
                 tc_fence_after();
                 const uint64_t dq0 = umma_desc(sbase + SL::kQ + cur_slot * SL::kTileBytes);
@@ -575,6 +609,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 tb.next(2);
                 if (nt < 2) ++nt;
               }
+              KVC_TR_SINCE(m_i, m_i0);
             }
             if (c.t == 0) qr.next(kQSlots);
             kr.next(SL::kStages);
@@ -582,6 +617,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           c.advance(P);
         }
       }
+      KVC_TR_PUT(3 + 6 * mine, m_q); KVC_TR_PUT(4 + 6 * mine, m_ko); KVC_TR_PUT(5 + 6 * mine, m_kx);
+      KVC_TR_PUT(6 + 6 * mine, m_t); KVC_TR_PUT(7 + 6 * mine, m_i); KVC_TR_PUT(8 + 6 * mine, KVC_TR_NOW() - m_s);
     }
   } else if (warp == 3) {
     // ============================== statistics exchange ========================================
@@ -675,6 +712,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
 
     int n1 = 0;
+    KVC_TR_DECL(e_t = 0, e_c = 0, e_b = 0, e_s = KVC_TR_NOW());
     float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
     bool ok = true;
 
@@ -714,7 +752,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       const int tile = c.tile();
       const bool run_ends = c.last(P);
       const int buf = n1 & 1;
-      if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word);
+      KVC_TR(e_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word));
       tc_fence_after();
       const long long c0 = (long long)tile * kTile + half * 64;
       const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;       // no masking anywhere in the tile
@@ -729,10 +767,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(buf));    // the accumulator is in registers now
-        if (ok && row_used) {
-          fast_chunk(ra);
-          fast_chunk(rb);
-        }
+        KVC_TR(e_c, if (ok && row_used) { fast_chunk(ra); fast_chunk(rb); });
       } else {
         float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
         p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
@@ -745,26 +780,26 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         // the two halves of every row meet through shared memory; the lower half's warps write
         // the run's record and report it to the statistics warp
         if (half == 1) *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
-        named_bar(3, 256);
+        KVC_TR(e_b, named_bar(3, 256));
         const float2 other = *stage;
-        named_bar(3, 256);                             // the stage may be written again
+        KVC_TR(e_b, named_bar(3, 256));                 // the stage may be written again
         if (half == 0) {
           float M = row_used ? mref : -INFINITY, Ls = row_used ? lsum : 0.f;
           combine(M, Ls, other.x, other.y);
           reinterpret_cast<float2*>(P.partial)[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
           __syncwarp();
           if (lane == 0) {
-            __threadfence();                            // this warp's part of the record, device-wide
-            const int seen = atomicAdd(reinterpret_cast<int*>(smem + SL::kFlushed), 1);
-            if ((seen & 3) == 3) {                      // the other three warps' parts are out as well
-              __threadfence();
-              red_add_release(P.group_counter + (long long)c.u * P.NG + c.j / kGroupRuns, 1);
-            }
+            // the four warps order their parts of the record through this counter (release /
+            // acquire within the CTA); the last one publishes the whole record with one
+            // device-wide release
+            const int seen = atom_add_acq_rel_cta_shared(sbase + SL::kFlushed, 1);
+            if ((seen & 3) == 3) red_add_release(P.group_counter + (long long)c.u * P.NG + c.j / kGroupRuns, 1);
           }
         }
         mref = -INFINITY; lsum = 0.f;
       }
     }
+    if (threadIdx.x == 256) { KVC_TR_PUT(15, e_t); KVC_TR_PUT(16, e_c); KVC_TR_PUT(17, KVC_TR_NOW() - e_s); KVC_TR_PUT(22, e_b); }
   } else {
     // ============================== pass-2 epilogue ============================================
     const int quarter = warp & 3;
@@ -775,6 +810,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const int n_chunks = (P.R + 31) / 32;
     int n2 = 0;
     bool ok = true;
+    KVC_TR_DECL(f_l = 0, f_t = 0, f_c = 0, f_s = KVC_TR_NOW());
 
     Cursor cu;
     cu.init(P);
@@ -784,29 +820,22 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       if (cu.t == 0) {
         // a new run: wait for its unit's log-sum-exp (the value itself is the flag)
         uint32_t bits = 0xffffffffu;
+        KVC_TR_DECL(f_l0 = KVC_TR_NOW());
         if (ok && trow < P.R) {
           const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
           bits = ld_relaxed_u32(src);
-          if (bits == 0xffffffffu) {
-            const unsigned long long t0 = globaltimer_ns();
-            uint32_t spins = 0;
-            while ((bits = ld_relaxed_u32(src)) == 0xffffffffu) {
-              __nanosleep(100);
-              if ((++spins & 255u) == 0) {
-                if (*abort_word) break;
-                if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
-              }
-            }
-          }
+          if (bits == 0xffffffffu) bits = poll_lse_slow(src, abort_word);
         }
         named_bar(1, 128);                             // everyone is done with the previous unit's values
         neg_lse[trow] = (trow < P.R) ? -__uint_as_float(bits) : 0.f;
         named_bar(1, 128);
+        KVC_TR_SINCE(f_l, f_l0);
         if (*abort_word) ok = false;
       }
       const int buf = 2 + (n2 & 1);
       const uint32_t tmem_col = (uint32_t)buf * kTile;
-      if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), abort_word);
+      KVC_TR(f_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), abort_word));
+      KVC_TR_DECL(f_c1 = KVC_TR_NOW());
       ++n2;
       tc_fence_after();
       const long long c = (long long)tile * kTile + trow;            // this thread's token
@@ -864,7 +893,9 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       }
       if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
       if (ok && c < P.N) P.scores[(long long)cu.u * P.N + c] = gacc;
+      KVC_TR_SINCE(f_c, f_c1);
     }
+    if (threadIdx.x == 128) { KVC_TR_PUT(18, f_l); KVC_TR_PUT(19, f_t); KVC_TR_PUT(20, f_c); KVC_TR_PUT(21, KVC_TR_NOW() - f_s); }
   }
 
   // ---------------- teardown ----------------
@@ -1038,3 +1069,10 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
 }
 
 }  // namespace kvc
+
+#ifdef KVC_SCORE_TRACE
+// Debug builds only: copies the trace counters (160 x 24 words) to the host.
+extern "C" __attribute__((visibility("default"))) int kvc_debug_dump(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, kvc::g_score_trace, sizeof(unsigned long long) * 160 * 24);
+}
+#endif
