@@ -39,13 +39,13 @@
 #include "kvc_internal.cuh"
 
 #ifndef KVC_SCORE_RUN_TILES
-#define KVC_SCORE_RUN_TILES 4      // tiles per run
+#define KVC_SCORE_RUN_TILES 8      // tiles per run
 #endif
 #ifndef KVC_SCORE_LAG_EXTRA
 #define KVC_SCORE_LAG_EXTRA 2      // runs of slack between a unit's last pass-1 run and its first pass-2 run
 #endif
 #ifndef KVC_SCORE_PREFETCH
-#define KVC_SCORE_PREFETCH 4       // pass-1 tiles prefetched into L2 ahead of their load
+#define KVC_SCORE_PREFETCH 2       // pass-1 tiles prefetched into L2 ahead of their load
 #endif
 
 namespace kvc {
