@@ -25,23 +25,47 @@ struct SelectState {
   unsigned long long rank;
 };
 
-// hist: [Bt][4][256] counts of digit (MSD first) among keys whose higher digits equal the prefix.
+// hist: [4][256] counts of digit (MSD first) among keys whose higher digits equal the prefix.
+// Walks the completed passes: in each, the digit whose cumulative count first reaches the rank.
+// Cooperative: the first 256 threads of the block take one bin each (blockDim.x >= 256); the
+// result is valid in every thread after the call.  `scratch` is 16 words of shared memory.
 __device__ inline SelectState derive_state(const unsigned int* __restrict__ hist_b, int passes,
-                                           unsigned long long rank0) {
+                                           unsigned long long rank0, unsigned long long* scratch) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   SelectState s;
   s.prefix = 0;
   s.rank = rank0;
   for (int p = 0; p < passes; ++p) {
-    const unsigned int* h = hist_b + p * kRadix;
-    unsigned long long cum = 0;
-    int dsel = kRadix - 1;
-    for (int dgt = 0; dgt < kRadix; ++dgt) {
-      const unsigned long long c = h[dgt];
-      if (cum + c >= s.rank) { dsel = dgt; break; }
-      cum += c;
+    unsigned long long c = 0, incl = 0;
+    if (tid < kRadix) {
+      c = hist_b[p * kRadix + tid];
+      incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (lane == 31) scratch[warp] = incl;
     }
-    s.rank -= cum;
-    s.prefix |= (uint32_t)dsel << (24 - 8 * p);
+    __syncthreads();
+    if (tid == 0) { scratch[8] = kRadix - 1; scratch[9] = 0; }     // default: the last digit
+    __syncthreads();
+    if (tid < kRadix) {
+      unsigned long long before = 0;
+      for (int wv = 0; wv < warp; ++wv) before += scratch[wv];
+      incl += before;
+      const unsigned long long excl = incl - c;
+      if (excl < s.rank && s.rank <= incl) { scratch[8] = (unsigned long long)tid; scratch[9] = excl; }
+    }
+    __syncthreads();
+    if (s.rank > 0) {
+      const unsigned long long total_last = scratch[9];
+      s.prefix |= (uint32_t)scratch[8] << (24 - 8 * p);
+      // when the rank lies beyond the total (cannot happen for a valid budget) the last digit
+      // was kept with nothing subtracted
+      s.rank -= total_last;
+    }
+    __syncthreads();
   }
   return s;
 }
@@ -50,11 +74,11 @@ __global__ void __launch_bounds__(kHistThreads)
 select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict__ hist, int pass,
                    int L, int Bt, long long N, long long budget) {
   __shared__ unsigned int sh[kRadix];
-  __shared__ SelectState st;
+  __shared__ unsigned long long scratch[16];
   const int b = blockIdx.y;
   unsigned int* hist_b = hist + (size_t)b * 4 * kRadix;
   for (int i = threadIdx.x; i < kRadix; i += kHistThreads) sh[i] = 0;
-  if (threadIdx.x == 0) st = derive_state(hist_b, pass, (unsigned long long)budget);
+  const SelectState st = derive_state(hist_b, pass, (unsigned long long)budget, scratch);
   __syncthreads();
   const uint32_t prefix = st.prefix;
   const int shift = 24 - 8 * pass;
@@ -77,37 +101,55 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
     if (sh[i]) atomicAdd(&hist_b[pass * kRadix + i], sh[i]);
 }
 
-// Number of entries of the non-increasing row with key < T (strictly better) and <= T.
-__device__ inline void count_layer(const float* __restrict__ row, long long N, uint32_t T,
-                                   long long* gt, long long* ge) {
-  long long lo = 0, hi = N;           // first index with key >= T
-  while (lo < hi) {
-    const long long mid = (lo + hi) >> 1;
-    if (score_to_key(row[mid]) < T) lo = mid + 1; else hi = mid;
+// One warp per layer: number of entries of the non-increasing row with key < T (strictly better)
+// and with key <= T, by a 32-way search (every step probes 32 positions at once).
+__device__ inline void count_layer_warp(const float* __restrict__ row, long long N, uint32_t T,
+                                        long long* gt, long long* ge) {
+  const int lane = threadIdx.x & 31;
+  // first index with key >= T, then first index with key > T: the same search with two predicates
+  long long res[2];
+#pragma unroll
+  for (int which = 0; which < 2; ++which) {
+    long long lo = 0, hi = N;                  // the answer lies in [lo, hi]
+    while (hi - lo > 0) {
+      const long long span = hi - lo;
+      const long long step = (span + 31) / 32;                 // probe lo + (lane + 1) * step - 1
+      const long long pos = lo + (lane + 1) * step - 1;
+      bool before = false;                                     // "row[pos] sorts before the boundary"
+      if (pos < hi) {
+        const uint32_t key = score_to_key(row[pos]);
+        before = which == 0 ? (key < T) : (key <= T);
+      }
+      const uint32_t m = __ballot_sync(0xffffffffu, before);   // a prefix of the lanes (the row is sorted)
+      const int n_before = __popc(m);
+      // the boundary lies after probe n_before - 1 and at or before probe n_before
+      const long long new_lo = n_before == 0 ? lo : min(hi, lo + (long long)n_before * step);
+      const long long new_hi = n_before == 32 ? hi : min(hi, lo + (long long)(n_before + 1) * step - 1);
+      lo = new_lo;
+      hi = new_hi;
+    }
+    res[which] = lo;
   }
-  *gt = lo;
-  hi = N;                              // first index with key > T
-  while (lo < hi) {
-    const long long mid = (lo + hi) >> 1;
-    if (score_to_key(row[mid]) <= T) lo = mid + 1; else hi = mid;
-  }
-  *ge = lo;
+  *gt = res[0];
+  *ge = res[1];
 }
 
-__global__ void select_finish_kernel(const float* __restrict__ composite,
-                                     const unsigned int* __restrict__ hist, int L, int Bt, long long N,
-                                     long long budget, int32_t* __restrict__ n_keep,
-                                     long long* __restrict__ offsets) {
+__global__ void __launch_bounds__(1024)
+select_finish_kernel(const float* __restrict__ composite,
+                     const unsigned int* __restrict__ hist, int L, int Bt, long long N,
+                     long long budget, int32_t* __restrict__ n_keep,
+                     long long* __restrict__ offsets) {
   __shared__ long long s_gt[KVC_MAX_LAYERS];
   __shared__ long long s_ge[KVC_MAX_LAYERS];
-  __shared__ uint32_t s_T;
+  __shared__ unsigned long long scratch[16];
   const int b = blockIdx.x;
-  if (threadIdx.x == 0) s_T = derive_state(hist + (size_t)b * 4 * kRadix, 4, (unsigned long long)budget).prefix;
-  __syncthreads();
-  const uint32_t T = s_T;
-  for (int l = threadIdx.x; l < L; l += blockDim.x) {
-    if (budget == 0) { s_gt[l] = 0; s_ge[l] = 0; }
-    else count_layer(composite + ((long long)l * Bt + b) * N, N, T, &s_gt[l], &s_ge[l]);
+  const SelectState st = derive_state(hist + (size_t)b * 4 * kRadix, 4, (unsigned long long)budget, scratch);
+  const uint32_t T = st.prefix;
+  const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int l = warp; l < L; l += n_warps) {
+    long long gt = 0, ge = 0;
+    if (budget > 0) count_layer_warp(composite + ((long long)l * Bt + b) * N, N, T, &gt, &ge);
+    if ((threadIdx.x & 31) == 0) { s_gt[l] = gt; s_ge[l] = ge; }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -156,7 +198,7 @@ kvc_status launch_allocate(const Problem& P, const float* composite, long long b
       KVC_LAUNCH_CHECK("select_hist_kernel");
     }
   }
-  select_finish_kernel<<<P.Bt, 128, 0, st>>>(composite, hist, P.L, P.Bt, P.N, budget, n_keep, offsets);
+  select_finish_kernel<<<P.Bt, 1024, 0, st>>>(composite, hist, P.L, P.Bt, P.N, budget, n_keep, offsets);
   KVC_LAUNCH_CHECK("select_finish_kernel");
   return KVC_OK;
 }
