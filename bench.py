@@ -228,6 +228,31 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def rank_workload(cfg, rank):
+    """Sequences are sharded over the ranks: rank r compresses its own sequence(s), drawn from seed r."""
+    return cfg.replace(seed=rank)
+
+
+def aggregate_tokens_per_s(cfg, world, ms_per_step):
+    """Whole-job throughput: every rank holds cfg.batch sequences of cfg.n_ctx context tokens."""
+    return cfg.batch * cfg.n_ctx * world / (ms_per_step * 1e-3)
+
+
+# DRAM traffic of one launch of the scoring kernel on the default workload, from the ncu capture
+# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of a 4-layer capture,
+# scaled by 8 to the 32 layers of the workload: the traffic is proportional to the layers).
+# None for any other workload, and to be reset to None whenever the kernel changes.
+SCORE_TRAFFIC_BYTES = {"llama8b_32k": None}
+
+
 def workload_config(cfg, world):
     return dict(workload=cfg.name, n_layers=cfg.n_layers, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                 head_dim=cfg.head_dim, n_ctx=cfg.n_ctx, window=cfg.window, batch_per_gpu=cfg.batch,
@@ -259,7 +284,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = pick_config(args).replace(seed=rank)
+    cfg = rank_workload(pick_config(args), rank)
     wl = W.make_workload(cfg, dev)
     desc = kvc.desc_from_config(cfg)
     budget = cfg.budget
@@ -350,16 +375,14 @@ def main():
         del hq, hk, hv, h_kout, h_vout
 
     # ---- max over ranks
-    t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0] + [stage_ms[n] for n in names], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
-    stage_ms = {n: float(t[2 + i]) for i, n in enumerate(names)}
+    t = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0] + [stage_ms[n] for n in names], dist, dev)
+    ms_total, e2e_ms = t[0], t[1]
+    stage_ms = {n: t[2 + i] for i, n in enumerate(names)}
 
     if rank == 0:
         ms_per_step = ms_total / args.steps
         tokens = cfg.batch * cfg.n_ctx * world
-        value = tokens / (ms_per_step * 1e-3)
+        value = aggregate_tokens_per_s(cfg, world, ms_per_step)
         peak, peak_kind = measured_peaks()
         ab = algorithmic_bytes(cfg)
         dominant = max(("score", "gather"), key=lambda n: stage_ms[n])
@@ -374,7 +397,8 @@ def main():
                                unit="GB/s", frac=ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
                                peak_kind=peak_kind, frac_of_8tbs=ab["total"] / (ms_per_step * 1e-3) / 8e12),
             roofline=dict(bound="hbm", kernel=dominant, achieved=ach, peak=peak, unit="GB/s", frac=ach / peak,
-                          traffic=None, peak_kind=peak_kind, algorithmic_bytes=ab[dominant]),
+                          traffic=SCORE_TRAFFIC_BYTES.get(cfg.name) if dominant == "score" else None,
+                          peak_kind=peak_kind, algorithmic_bytes=ab[dominant]),
         )
         if e2e:
             line["e2e"] = dict(value=tokens / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=e2e["h2d"],

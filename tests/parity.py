@@ -105,7 +105,7 @@ def assert_gather_exact(wl, desc, idx_gpu, n_keep, offsets, k_out, v_out, layers
             n = int(n_keep[b, l])
             lo = int(offsets[b, l]) * Hkv * d
             for (src, dst, name) in ((wl.k, ko, "K"), (wl.v, vo, "V")):
-                ref = oracle.gather_layer(raw_numpy(src[l][b]), idx_gpu[l, b], n)
+                ref = oracle.gather_layer(raw_numpy(src[l][b]), idx_gpu[l][b], n)
                 got = dst[b, lo:lo + Hkv * n * d].reshape(Hkv, n, d)
                 assert np.array_equal(ref, got), "%s' differs at layer %d seq %d" % (name, l, b)
 
