@@ -86,14 +86,18 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
   const long long total = (long long)L * N;
   const long long tile = (long long)kHistThreads * kItemsPerThread;
   for (long long t0 = (long long)blockIdx.x * tile; t0 < total; t0 += (long long)gridDim.x * tile) {
+    // pooled index -> (layer, position) once per tile, then by steps of the block width
+    long long i = t0 + threadIdx.x;
+    long long l = i / N, kk = i - l * N;
 #pragma unroll 4
     for (int it = 0; it < kItemsPerThread; ++it) {
-      const long long i = t0 + (long long)it * kHistThreads + threadIdx.x;
       if (i < total) {
-        const long long l = i / N, kk = i - l * N;
         const uint32_t key = score_to_key(composite[(l * Bt + b) * N + kk]);
         if ((key & hi_mask) == prefix) atomicAdd(&sh[(key >> shift) & 0xffu], 1u);
       }
+      i += kHistThreads;
+      kk += kHistThreads;
+      while (kk >= N) { kk -= N; ++l; }
     }
   }
   __syncthreads();
