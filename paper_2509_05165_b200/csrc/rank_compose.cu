@@ -2,22 +2,25 @@
 //
 // Every (layer, sequence, KV head) is one segment of N (score, position) pairs that must come
 // out in descending score order with equal scores in ascending position.  Scores are mapped to
-// 32-bit keys whose ascending order is the wanted order, and each segment is sorted by one CTA
-// with a stable least-significant-digit radix sort (8-bit digits, 4 passes, tiles of 8192
-// elements with eight per thread so that the loads of a tile are in flight together) that
-// ping-pongs between two scratch buffers; a segment's working set (8 bytes per token per buffer)
-// stays in L2 between passes.  The last pass writes the positions straight into idx and leaves the sorted
-// keys for the composite kernel, which turns them back into scores and reduces over the heads.
+// 32-bit keys whose ascending order is the wanted order, and all segments are sorted together by
+// a stable least-significant-digit radix sort (8-bit digits, 4 passes) over tiles of 4096
+// elements.  A pass is two kernels: one counts the digit of every tile, the other gives every
+// tile its own CTA, which derives the tile's output ranges from the counts of its segment,
+// ranks its elements, reorders them by digit in shared memory and writes them out in runs.
+// Tiles are independent inside a pass, so the whole GPU is busy whatever the number of
+// segments; the passes ping-pong between two scratch buffers that stay in L2.  The last pass
+// writes the positions straight into idx and leaves the sorted keys for the composite kernel,
+// which turns them back into scores and reduces over the heads.
 #include "kvc_internal.cuh"
 
 namespace kvc {
 namespace {
 
-constexpr int kSortThreads = 512;            // two CTAs per SM: all 256 segments of the 8B shape are resident at once
+constexpr int kSortThreads = 512;
 constexpr int kWarps = kSortThreads / 32;
 constexpr int kRadix = 256;
-constexpr int kItems = 8;                               // elements per thread per tile
-constexpr int kTileItems = kSortThreads * kItems;       // 8192 elements per tile
+constexpr int kItems = 8;                               // elements per thread
+constexpr int kTileItems = kSortThreads * kItems;       // 4096 elements per tile
 constexpr int kWarpItems = 32 * kItems;                 // a warp owns 256 consecutive elements of a tile
 
 struct SortBuffers {
@@ -38,168 +41,166 @@ __device__ __forceinline__ uint32_t same_digit_lanes(uint32_t digit, bool valid)
   return valid ? peers : 0u;
 }
 
-__global__ void __launch_bounds__(kSortThreads, 2)
-segment_sort_kernel(const float* __restrict__ scores, int32_t* __restrict__ idx_out,
-                    SortBuffers buf, long long N) {
-  __shared__ uint32_t hist4[4][kRadix];
-  __shared__ uint32_t base[kRadix];               // running start of every digit's output range
-  __shared__ uint32_t tile_base[kRadix];          // ... as it was when the current tile began
-  __shared__ uint16_t warp_cnt[kWarps][kRadix];   // per tile: count, then exclusive offset, per (warp, digit)
-  __shared__ uint32_t scan_tmp[kRadix / 32];
-  __shared__ uint32_t tile_start[kRadix];         // first slot of every digit inside the reordered tile
-  __shared__ uint32_t stage_k[kTileItems];        // the tile, reordered by digit, before it goes out
-  __shared__ int32_t stage_v[kTileItems];
+// Source and destination of a pass.  0: scores -> A;  1: A -> B;  2: B -> A;  3: A -> (keys_b, idx).
+struct PassIo {
+  const uint32_t* src_k; const int32_t* src_v;
+  uint32_t* dst_k; int32_t* dst_v;
+};
+__device__ __forceinline__ PassIo pass_io(const SortBuffers& buf, int32_t* idx_out, int pass, long long seg_off) {
+  PassIo io;
+  io.src_k = ((pass == 2) ? buf.keys_b : buf.keys_a) + seg_off;
+  io.src_v = ((pass == 2) ? buf.vals_b : buf.vals_a) + seg_off;
+  io.dst_k = ((pass == 0 || pass == 2) ? buf.keys_a : buf.keys_b) + seg_off;
+  io.dst_v = ((pass == 0 || pass == 2) ? buf.vals_a : (pass == 3 ? idx_out : buf.vals_b)) + seg_off;
+  return io;
+}
 
-  const long long seg = blockIdx.x;
+// counts[seg][tile][digit]: how many elements of the tile have that digit in this pass.
+__global__ void __launch_bounds__(kSortThreads)
+sort_count_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
+                  uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
+  __shared__ uint32_t hist[kRadix];
+  const long long seg = blockIdx.x / tiles;
+  const int tile = (int)(blockIdx.x - seg * tiles);
+  const PassIo io = pass_io(buf, idx_out, pass, seg * N);
   const float* s_in = scores + seg * N;
-  uint32_t* ka = buf.keys_a + seg * N; int32_t* va = buf.vals_a + seg * N;
-  uint32_t* kb = buf.keys_b + seg * N; int32_t* vb = buf.vals_b + seg * N;
-  int32_t* out_idx = idx_out + seg * N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
-
-  // ---- digit histograms of all four passes in one sweep (the multiset of keys never changes)
-  for (int i = tid; i < 4 * kRadix; i += kSortThreads) (&hist4[0][0])[i] = 0;
+  const int shift = 8 * pass;
+  for (int i = tid; i < kRadix; i += kSortThreads) hist[i] = 0;
   __syncthreads();
-  for (long long t0 = 0; t0 < N; t0 += kTileItems) {
-    uint32_t key[kItems];
-    bool valid[kItems];
+  const long long w0 = (long long)tile * kTileItems + (long long)warp * kWarpItems;
 #pragma unroll
-    for (int k = 0; k < kItems; ++k) {
-      const long long i = t0 + (long long)warp * kWarpItems + k * 32 + lane;
-      valid[k] = i < N;
-      key[k] = valid[k] ? score_to_key(s_in[i]) : 0u;
-    }
-#pragma unroll
-    for (int k = 0; k < kItems; ++k) {
-      // the three low digits are spread over their 256 bins: plain shared-memory atomics hardly
-      // collide.  The top digit (sign and high exponent bits) takes a handful of values, so the
-      // warp adds its lanes up first.
-#pragma unroll
-      for (int pass = 0; pass < 3; ++pass)
-        if (valid[k]) atomicAdd(&hist4[pass][(key[k] >> (8 * pass)) & 0xffu], 1u);
-      const uint32_t digit = key[k] >> 24;
-      const uint32_t peers = same_digit_lanes(digit, valid[k]);
-      if (valid[k] && (peers & lt_mask) == 0) atomicAdd(&hist4[3][digit], (uint32_t)__popc(peers));
+  for (int k = 0; k < kItems; ++k) {
+    const long long i = w0 + k * 32 + lane;
+    const bool valid = i < N;
+    uint32_t key = 0;
+    if (valid) key = (pass == 0) ? score_to_key(s_in[i]) : io.src_k[i];
+    const uint32_t digit = (key >> shift) & 0xffu;
+    if (pass < 3) {
+      // the low digits are spread over their 256 bins: plain shared-memory atomics hardly collide
+      if (valid) atomicAdd(&hist[digit], 1u);
+    } else {
+      // the top digit (sign and high exponent bits) takes a handful of values: add up per warp first
+      const uint32_t peers = same_digit_lanes(digit, valid);
+      if (valid && (peers & lt_mask) == 0) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
     }
   }
   __syncthreads();
+  for (int i = tid; i < kRadix; i += kSortThreads) counts[((long long)seg * tiles + tile) * kRadix + i] = hist[i];
+}
 
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 8 * pass;
-    // pass 0: scores -> A;  1: A -> B;  2: B -> A;  3: A -> (keys_b, idx)
-    const uint32_t* src_k = (pass == 2) ? kb : ka;
-    const int32_t* src_v = (pass == 2) ? vb : va;
-    uint32_t* dst_k = (pass == 0 || pass == 2) ? ka : kb;
-    int32_t* dst_v = (pass == 0 || pass == 2) ? va : (pass == 3 ? out_idx : vb);
-    const uint32_t* hist = hist4[pass];
+// One tile of one pass: stable scatter.  Inside a tile the order is (warp, item, lane), which
+// is the order of the positions.
+__global__ void __launch_bounds__(kSortThreads, 2)
+sort_scatter_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
+                    const uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
+  __shared__ uint32_t tile_base[kRadix];          // first output position of every digit for this tile
+  __shared__ uint32_t tile_start[kRadix];         // first slot of every digit inside the reordered tile
+  __shared__ uint16_t warp_cnt[kWarps][kRadix];   // count, then exclusive offset, per (warp, digit)
+  __shared__ uint32_t scan_tmp[2][kRadix / 32];
+  __shared__ uint32_t stage_k[kTileItems];        // the tile, reordered by digit, before it goes out
+  __shared__ int32_t stage_v[kTileItems];
 
-    // ---- exclusive scan of the 256 bins -> base
-    if (tid < kRadix) {
-      const uint32_t v = hist[tid];
-      uint32_t incl = v;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
-      }
-      if (lane == 31) scan_tmp[warp] = incl;
-      base[tid] = incl - v;
-    }
-    __syncthreads();
-    if (tid < kRadix) {
-      uint32_t add = 0;
-      for (int wv = 0; wv < warp; ++wv) add += scan_tmp[wv];
-      base[tid] += add;
-    }
-    __syncthreads();
+  const long long seg = blockIdx.x / tiles;
+  const int tile = (int)(blockIdx.x - seg * tiles);
+  const PassIo io = pass_io(buf, idx_out, pass, seg * N);
+  const float* s_in = scores + seg * N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  const int shift = 8 * pass;
+  const long long t0 = (long long)tile * kTileItems;
 
-    // ---- stable scatter, one tile of 8192 elements at a time, tiles in order.  Inside a tile
-    //      the order is (warp, item, lane), which is the order of the positions.
-    for (long long t0 = 0; t0 < N; t0 += kTileItems) {
-      uint32_t key[kItems]; int32_t val[kItems]; uint32_t rank[kItems];
-      const long long w0 = t0 + (long long)warp * kWarpItems;
+  // ---- the tile's elements (issued first: the loads are in flight during the prologue)
+  uint32_t key[kItems]; int32_t val[kItems]; uint32_t rank[kItems];
+  {
+    const long long w0 = t0 + (long long)warp * kWarpItems;
 #pragma unroll
-      for (int k = 0; k < kItems; ++k) {
-        const long long i = w0 + k * 32 + lane;
-        key[k] = 0; val[k] = -1;
-        if (i < N) {
-          if (pass == 0) { key[k] = score_to_key(s_in[i]); val[k] = (int32_t)i; }
-          else { key[k] = src_k[i]; val[k] = src_v[i]; }
-        }
+    for (int k = 0; k < kItems; ++k) {
+      const long long i = w0 + k * 32 + lane;
+      key[k] = 0; val[k] = -1;
+      if (i < N) {
+        if (pass == 0) { key[k] = score_to_key(s_in[i]); val[k] = (int32_t)i; }
+        else { key[k] = io.src_k[i]; val[k] = io.src_v[i]; }
       }
-      // this warp's counters, then the rank of every item among the warp's items of its digit
-      for (int dgt = lane; dgt < kRadix; dgt += 32) warp_cnt[warp][dgt] = 0;
-      __syncwarp();
-#pragma unroll
-      for (int k = 0; k < kItems; ++k) {
-        const bool valid = val[k] >= 0;
-        const uint32_t digit = (key[k] >> shift) & 0xffu;
-        const uint32_t peers = same_digit_lanes(digit, valid);
-        uint32_t before = 0;
-        if (valid) before = warp_cnt[warp][digit];
-        __syncwarp();
-        if (valid && (peers & lt_mask) == 0) warp_cnt[warp][digit] = (uint16_t)(before + __popc(peers));
-        __syncwarp();
-        rank[k] = before + __popc(peers & lt_mask);
-      }
-      __syncthreads();
-      // per digit: exclusive scan over the warps; then the digit's first slot inside the tile
-      // (exclusive scan over the digits) and its first position in the output
-      uint32_t run = 0, incl = 0;
-      if (tid < kRadix) {
-#pragma unroll 8
-        for (int wv = 0; wv < kWarps; ++wv) {
-          const uint32_t cnt = warp_cnt[wv][tid];
-          warp_cnt[wv][tid] = (uint16_t)run;
-          run += cnt;
-        }
-        incl = run;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += n;
-        }
-        if (lane == 31) scan_tmp[warp] = incl;
-      }
-      __syncthreads();
-      if (tid < kRadix) {
-        uint32_t add = 0;
-        for (int wv = 0; wv < warp; ++wv) add += scan_tmp[wv];
-        tile_start[tid] = incl - run + add;
-        tile_base[tid] = base[tid];
-        base[tid] += run;
-      }
-      __syncthreads();
-      // reorder the tile by digit in shared memory ...
-#pragma unroll
-      for (int k = 0; k < kItems; ++k) {
-        if (val[k] >= 0) {
-          const uint32_t digit = (key[k] >> shift) & 0xffu;
-          const uint32_t slot = tile_start[digit] + warp_cnt[warp][digit] + rank[k];
-          stage_k[slot] = key[k];
-          stage_v[slot] = val[k];
-        }
-      }
-      __syncthreads();
-      // ... and write it out: neighbouring threads hold neighbours of the same digit, so the
-      // stores of a warp fall into a few contiguous runs
-      const int n_tile = (int)min((long long)kTileItems, N - t0);
-#pragma unroll
-      for (int k = 0; k < kItems; ++k) {
-        const int slot = k * kSortThreads + tid;
-        if (slot < n_tile) {
-          const uint32_t kk = stage_k[slot];
-          const uint32_t digit = (kk >> shift) & 0xffu;
-          const uint32_t pos = tile_base[digit] + ((uint32_t)slot - tile_start[digit]);
-          dst_k[pos] = kk;
-          dst_v[pos] = stage_v[slot];
-        }
-      }
-      __syncthreads();      // the stage and the per-tile tables are reused by the next tile
     }
-    __threadfence_block();
-    __syncthreads();
+  }
+
+  // ---- where the tile's digits go: (elements of smaller digits in the whole segment) +
+  //      (elements of the same digit in earlier tiles); and where they sit inside the tile
+  uint32_t total = 0, before = 0, mine = 0, incl_t = 0, incl_m = 0;
+  if (tid < kRadix) {
+    const uint32_t* c = counts + (long long)seg * tiles * kRadix + tid;
+    for (int t = 0; t < tiles; ++t) {
+      const uint32_t v = c[(long long)t * kRadix];
+      total += v;
+      if (t < tile) before += v;
+      if (t == tile) mine = v;
+    }
+    incl_t = total; incl_m = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t a = __shfl_up_sync(0xffffffffu, incl_t, o);
+      const uint32_t b2 = __shfl_up_sync(0xffffffffu, incl_m, o);
+      if (lane >= o) { incl_t += a; incl_m += b2; }
+    }
+    if (lane == 31) { scan_tmp[0][warp] = incl_t; scan_tmp[1][warp] = incl_m; }
+  }
+  // this warp's counters, then the rank of every element among the warp's elements of its digit
+  for (int dgt = lane; dgt < kRadix; dgt += 32) warp_cnt[warp][dgt] = 0;
+  __syncwarp();
+#pragma unroll
+  for (int k = 0; k < kItems; ++k) {
+    const bool valid = val[k] >= 0;
+    const uint32_t digit = (key[k] >> shift) & 0xffu;
+    const uint32_t peers = same_digit_lanes(digit, valid);
+    uint32_t seen = 0;
+    if (valid) seen = warp_cnt[warp][digit];
+    __syncwarp();
+    if (valid && (peers & lt_mask) == 0) warp_cnt[warp][digit] = (uint16_t)(seen + __popc(peers));
+    __syncwarp();
+    rank[k] = seen + __popc(peers & lt_mask);
+  }
+  __syncthreads();
+  if (tid < kRadix) {
+    uint32_t add_t = 0, add_m = 0;
+    for (int wv = 0; wv < warp; ++wv) { add_t += scan_tmp[0][wv]; add_m += scan_tmp[1][wv]; }
+    tile_base[tid] = incl_t - total + add_t + before;
+    tile_start[tid] = incl_m - mine + add_m;
+    // per digit: exclusive scan over the warps
+    uint32_t run = 0;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) {
+      const uint32_t cnt = warp_cnt[wv][tid];
+      warp_cnt[wv][tid] = (uint16_t)run;
+      run += cnt;
+    }
+  }
+  __syncthreads();
+  // ---- reorder the tile by digit in shared memory ...
+#pragma unroll
+  for (int k = 0; k < kItems; ++k) {
+    if (val[k] >= 0) {
+      const uint32_t digit = (key[k] >> shift) & 0xffu;
+      const uint32_t slot = tile_start[digit] + warp_cnt[warp][digit] + rank[k];
+      stage_k[slot] = key[k];
+      stage_v[slot] = val[k];
+    }
+  }
+  __syncthreads();
+  // ---- ... and write it out: neighbouring threads hold neighbours of the same digit, so the
+  //      stores of a warp fall into a few contiguous runs
+  const int n_tile = (int)min((long long)kTileItems, N - t0);
+#pragma unroll
+  for (int k = 0; k < kItems; ++k) {
+    const int slot = k * kSortThreads + tid;
+    if (slot < n_tile) {
+      const uint32_t kk = stage_k[slot];
+      const uint32_t digit = (kk >> shift) & 0xffu;
+      const uint32_t pos = tile_base[digit] + ((uint32_t)slot - tile_start[digit]);
+      io.dst_k[pos] = kk;
+      io.dst_v[pos] = stage_v[slot];
+    }
   }
 }
 
@@ -222,9 +223,12 @@ __global__ void compose_kernel(const uint32_t* __restrict__ keys, float* __restr
 
 }  // namespace
 
+static int sort_tiles(const Problem& P) { return (int)((P.N + kTileItems - 1) / kTileItems); }
+
 size_t compose_workspace_bytes(const Problem& P) {
   const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
-  return 4 * align_up(items * 4);
+  const size_t segments = (size_t)P.L * P.Bt * P.Hkv;
+  return 4 * align_up(items * 4) + align_up(segments * sort_tiles(P) * kRadix * sizeof(uint32_t));
 }
 
 kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, float* composite,
@@ -241,9 +245,20 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
   buf.vals_a = reinterpret_cast<int32_t*>(w + region);
   buf.keys_b = reinterpret_cast<uint32_t*>(w + 2 * region);
   buf.vals_b = reinterpret_cast<int32_t*>(w + 3 * region);
+  uint32_t* counts = reinterpret_cast<uint32_t*>(w + 4 * region);
   const long long segments = (long long)P.L * P.Bt * P.Hkv;
-  segment_sort_kernel<<<(unsigned)segments, kSortThreads, 0, st>>>(scores, idx, buf, P.N);
-  KVC_LAUNCH_CHECK("segment_sort_kernel");
+  const int tiles = sort_tiles(P);
+  const long long blocks = segments * tiles;
+  if (blocks >= (1LL << 31)) {
+    set_error("compose: too many sort tiles");
+    return KVC_ERR_UNSUPPORTED;
+  }
+  for (int pass = 0; pass < 4; ++pass) {
+    sort_count_kernel<<<(unsigned)blocks, kSortThreads, 0, st>>>(scores, buf, idx, counts, P.N, tiles, pass);
+    KVC_LAUNCH_CHECK("sort_count_kernel");
+    sort_scatter_kernel<<<(unsigned)blocks, kSortThreads, 0, st>>>(scores, buf, idx, counts, P.N, tiles, pass);
+    KVC_LAUNCH_CHECK("sort_scatter_kernel");
+  }
   const long long total = (long long)P.L * P.Bt * P.N;
   compose_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(buf.keys_b, composite, P.Hkv, P.N,
                                                                  total, P.agg_head);
