@@ -56,7 +56,7 @@ __device__ __forceinline__ PassIo pass_io(const SortBuffers& buf, int32_t* idx_o
 }
 
 // counts[seg][tile][digit]: how many elements of the tile have that digit in this pass.
-__global__ void __launch_bounds__(kSortThreads)
+__global__ void __launch_bounds__(kSortThreads, 4)
 sort_count_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
                   uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
   __shared__ uint32_t hist[kRadix];
