@@ -38,8 +38,10 @@ size_t score_workspace_bytes(const Problem& P) {
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
                         float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
   if (score_sm100_supported(P)) {
-    const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st);
-    if (s == KVC_OK) return launch_score_augment(P, scores, st);
+    const float* parts = nullptr;
+    int row_tiles = 1;
+    const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st, &parts, &row_tiles);
+    if (s == KVC_OK) return launch_score_augment(P, scores, parts, row_tiles, st);
     if (s != KVC_ERR_UNSUPPORTED) return s;      // a real failure; UNSUPPORTED = strides TMA cannot take
   }
   return launch_score_generic(P, gm, q, k, scores, ws, ws_bytes, st);

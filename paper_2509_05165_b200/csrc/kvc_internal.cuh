@@ -66,17 +66,21 @@ size_t score_workspace_bytes(const Problem& P);
 // Eqs. 3, 14-16: writes scores [L, Bt, Hkv, N].
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
                         float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
-// The two implementations behind it: CUDA cores (any supported shape) and tcgen05 (bf16, GQA
-// groups of up to 128 window rows).
+// The two implementations behind it: CUDA cores (any supported shape) and tcgen05 (bf16,
+// contiguous GQA groups, window of 8, 16, 32, 64 or 128 rows).
 size_t score_generic_workspace_bytes(const Problem& P);
 kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
                                 const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,
                                 cudaStream_t st);
-kvc_status launch_score_augment(const Problem& P, float* scores, cudaStream_t st);
+// Eq. 16 in place; before it, with `row_tiles` > 1, the group aggregate (Eq. 15) of every KV head
+// from its row tiles' partial aggregates `parts` [row_tiles][L*Bt*Hkv][N], in tile order.
+kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
+                                cudaStream_t st);
 bool score_sm100_supported(const Problem& P);
 size_t score_sm100_workspace_bytes(const Problem& P);
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
-                              int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
+                              int* device_status, void* ws, size_t ws_bytes, cudaStream_t st,
+                              const float** parts_out, int* row_tiles_out);
 
 // ---- rank + compose ---------------------------------------------------------------------------
 size_t compose_workspace_bytes(const Problem& P);

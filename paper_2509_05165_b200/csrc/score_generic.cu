@@ -239,12 +239,28 @@ score_emit_kernel(ScoreParams P, GroupMap gm, LayerPtrs qp, LayerPtrs kp,
   if (valid) s_group[((long long)lb * P.Hkv + h) * P.N + c] = gacc;
 }
 
-// Eq. 16: S[h, c] = S_group[h, c] + (1/Hkv) sum_i S_group[i, c], in place.
-__global__ void score_augment_kernel(float* __restrict__ s, int Hkv, long long N, long long total) {
+// Eq. 16: S[h, c] = S_group[h, c] + (1/Hkv) sum_i S_group[i, c], in place.  With row tiles, first
+// Eq. 15 from the tiles' partial aggregates (sum or max over the tile's query heads), in tile order.
+__global__ void score_augment_kernel(float* __restrict__ s, const float* __restrict__ parts, int row_tiles,
+                                     int G, int agg_group, int augment, int Hkv, long long N, long long total) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const long long lb = i / N, c = i - lb * N;
   float* base = s + lb * Hkv * N + c;
+  if (row_tiles > 1) {
+    const long long tile_stride = (total / N) * Hkv * N;          // one [L*Bt*Hkv][N] block per row tile
+    const float* pbase = parts + lb * Hkv * N + c;
+    for (int h = 0; h < Hkv; ++h) {
+      float acc = pbase[(long long)h * N];
+      for (int t = 1; t < row_tiles; ++t) {
+        const float v = pbase[(long long)t * tile_stride + (long long)h * N];
+        acc = (agg_group == KVC_AGG_MAX) ? fmaxf(acc, v) : acc + v;
+      }
+      if (agg_group == KVC_AGG_MEAN) acc = acc / (float)G;
+      base[(long long)h * N] = acc;
+    }
+  }
+  if (!augment) return;
   float sum = 0.f;
   for (int h = 0; h < Hkv; ++h) sum += base[(long long)h * N];
   const float mean = sum / (float)Hkv;
@@ -289,10 +305,12 @@ size_t score_generic_workspace_bytes(const Problem& P) {
   return align_up(rows * generic_nchunks(P) * sizeof(float2)) + align_up(rows * sizeof(float));
 }
 
-kvc_status launch_score_augment(const Problem& P, float* scores, cudaStream_t st) {
-  if (!P.augment) return KVC_OK;
+kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
+                                cudaStream_t st) {
+  if (!P.augment && row_tiles <= 1) return KVC_OK;
   const long long total = (long long)P.L * P.Bt * P.N;
-  score_augment_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(scores, P.Hkv, P.N, total);
+  score_augment_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+      scores, parts, row_tiles, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total);
   KVC_LAUNCH_CHECK("score_augment_kernel");
   return KVC_OK;
 }
@@ -318,7 +336,7 @@ kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const Laye
     else s = run<float, 128>(P, gm, q, k, scores, partial, lse2, nchunks, st);
   }
   if (s != KVC_OK) return s;
-  return launch_score_augment(P, scores, st);
+  return launch_score_augment(P, scores, nullptr, 1, st);
 }
 
 }  // namespace kvc

@@ -22,6 +22,11 @@
 //                        the score store is coalesced.  max_m exp(s_m - lse_m) is evaluated as
 //                        exp(max_m(s_m - lse_m)): one exponential per query head, not per row.
 //
+// A unit is a (layer, sequence, KV head, row tile): the G x w window rows of a KV head are cut
+// into row tiles of at most 128 rows (whole query heads), so that any GQA group / window size
+// with w <= 128 runs here; with more than one row tile the pass-2 results are partial group
+// aggregates that the Eq. 16 kernel combines in a fixed order.
+//
 // Every CTA walks one static sequence that alternates a pass-1 tile with a pass-2 tile; the
 // pass-2 stream trails the pass-1 stream by `shift` tiles.  A pass-2 tile only ever waits for
 // pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot deadlock while all
@@ -88,12 +93,13 @@ struct FastParams {
   int* unit_counter;           // [U], preset to -1
   unsigned int* lse2;          // [U][128] fp32 bits, preset to 0xffffffff ("not there yet")
   int* status;                 // device status word (may be null)
-  float* scores;               // [U][N]
-  int L, Bt, Hkv, G, R;
+  float* scores;               // [L*Bt*Hkv][N], or with QT > 1 the partial aggregates [QT][L*Bt*Hkv][N]
+  int L, Bt, Hkv, G;
+  int HPT, QT, w;              // query heads per row tile, row tiles per KV head, window rows per query head
   long long N, q_pos0;
   int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
   int step_u, step_j;          // grid = step_u * RPU + step_j: how a CTA's next run moves (unit, run in unit)
-  int step_l, step_b, step_h;  // step_u = (step_l * Bt + step_b) * Hkv + step_h
+  int step_l, step_b, step_h, step_q;  // step_u = ((step_l * Bt + step_b) * Hkv + step_h) * QT + step_q
   unsigned int total_runs;     // U * RPU
   int shift;                   // tiles by which the pass-2 stream trails the pass-1 stream
   float sl2e;                  // scale * log2(e)
@@ -285,16 +291,22 @@ __device__ __forceinline__ void combine(float& M, float& Ls, float m, float l) {
 struct Cursor {
   int t;            // position inside the run, 0 .. kRunTiles-1
   int u, j;         // unit, run inside the unit
-  int l, b, h;      // the unit's layer, sequence, KV head
+  int l, b, h, q;   // the unit's layer, sequence, KV head, row tile
   __device__ __forceinline__ void init(const FastParams& P) {
     t = 0;
     u = (int)(blockIdx.x / (unsigned int)P.RPU);
     j = (int)(blockIdx.x - (unsigned int)u * (unsigned int)P.RPU);
-    const int lb = u / P.Hkv;
-    h = u - lb * P.Hkv;
+    const int uh = u / P.QT;
+    q = u - uh * P.QT;
+    const int lb = uh / P.Hkv;
+    h = uh - lb * P.Hkv;
     l = lb / P.Bt;
     b = lb - l * P.Bt;
   }
+  // window rows of this unit's row tile (whole query heads; the last tile of a KV head may be short)
+  __device__ __forceinline__ int rows(const FastParams& P) const { return min(P.HPT, P.G - q * P.HPT) * P.w; }
+  // index of the (layer, sequence, KV head)
+  __device__ __forceinline__ int kv_unit(const FastParams& P) const { return (l * P.Bt + b) * P.Hkv + h; }
   __device__ __forceinline__ int tile() const { return j * kRunTiles + t; }
   __device__ __forceinline__ bool valid(const FastParams& P) const { return tile() < P.NT; }
   // last valid tile of its run
@@ -304,6 +316,8 @@ struct Cursor {
     int c = 0;
     if (j >= P.RPU) { j -= P.RPU; c = 1; }
     u += P.step_u + c;
+    q += P.step_q + c; c = 0;
+    if (q >= P.QT) { q -= P.QT; c = 1; }
     h += P.step_h + c; c = 0;
     if (h >= P.Hkv) { h -= P.Hkv; c = 1; }
     b += P.step_b + c; c = 0;
@@ -479,7 +493,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   const int my_runs = (P.total_runs > blockIdx.x) ? (int)((P.total_runs - blockIdx.x + P.grid - 1) / P.grid) : 0;
   const int my_tiles = my_runs * kRunTiles;                  // stream length (some positions hold no tile)
   const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
-  const uint32_t q_bytes = (uint32_t)P.R * D * 2;
+  const uint32_t q_bytes = (uint32_t)(P.HPT * P.w) * D * 2;   // the whole box arrives (rows outside the tensor as zeros)
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
   if (warp == 0) {
@@ -518,7 +532,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 mbar_expect_tx(bar_qfull(qr.i), q_bytes);
                 for (int hf = 0; hf < SL::kHalves; ++hf)
                   tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
-                              bar_qfull(qr.i), hf * 64, 0, c.h * P.G, c.b, pol_keep);
+                              bar_qfull(qr.i), hf * 64, 0, c.h * P.G + c.q * P.HPT, c.b, pol_keep);
                 qr.next(kQSlots);
                 if (qc < kQSlots) ++qc;
               }
@@ -705,7 +719,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const int half = (warp - 8) >> 2;                 // which 64 columns (tokens) of every tile
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;              // TMEM lane = query row
-    const bool row_used = row < P.R;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + row;
     const long long row_vis = min(P.N - 1, P.q_pos0 + (row % W));     // last key this row sees
@@ -751,6 +764,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       if (!c.valid(P)) continue;
       const int tile = c.tile();
       const bool run_ends = c.last(P);
+      const bool row_used = row < c.rows(P);
       const int buf = n1 & 1;
       KVC_TR(e_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word));
       tc_fence_after();
@@ -807,7 +821,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float* neg_lse = reinterpret_cast<float*>(smem + SL::kNegLse);
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
-    const int n_chunks = (P.R + 31) / 32;
     int n2 = 0;
     bool ok = true;
     KVC_TR_DECL(f_l = 0, f_t = 0, f_c = 0, f_s = KVC_TR_NOW());
@@ -817,17 +830,19 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     for (int idx = 0; idx < my_tiles; ++idx, cu.advance(P)) {
       if (!cu.valid(P)) continue;
       const int tile = cu.tile();
+      const int rows_u = cu.rows(P);
+      const int n_chunks = (rows_u + 31) / 32;
       if (cu.t == 0) {
         // a new run: wait for its unit's log-sum-exp (the value itself is the flag)
         uint32_t bits = 0xffffffffu;
         KVC_TR_DECL(f_l0 = KVC_TR_NOW());
-        if (ok && trow < P.R) {
+        if (ok && trow < rows_u) {
           const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
           bits = ld_relaxed_u32(src);
           if (bits == 0xffffffffu) bits = poll_lse_slow(src, abort_word);
         }
         named_bar(1, 128);                             // everyone is done with the previous unit's values
-        neg_lse[trow] = (trow < P.R) ? -__uint_as_float(bits) : 0.f;
+        neg_lse[trow] = (trow < rows_u) ? -__uint_as_float(bits) : 0.f;
         named_bar(1, 128);
         KVC_TR_SINCE(f_l, f_l0);
         if (*abort_word) ok = false;
@@ -885,14 +900,16 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           }
         }
       } else {
-        gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, P.R, P.sl2e, full,
+        gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
                                              c - P.q_pos0, P.agg_group);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(buf));
       }
-      if (P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
-      if (ok && c < P.N) P.scores[(long long)cu.u * P.N + c] = gacc;
+      // one row tile: the group aggregate itself; several: this tile's part of it
+      if (P.QT == 1 && P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
+      if (ok && c < P.N)
+        P.scores[((long long)cu.q * ((long long)P.L * P.Bt * P.Hkv) + cu.kv_unit(P)) * P.N + c] = gacc;
       KVC_TR_SINCE(f_c, f_c1);
     }
     if (threadIdx.x == 128) { KVC_TR_PUT(18, f_l); KVC_TR_PUT(19, f_t); KVC_TR_PUT(20, f_c); KVC_TR_PUT(21, KVC_TR_NOW() - f_s); }
@@ -943,13 +960,17 @@ bool encode_map(CUtensorMap* m, const void* base, const long long dims[4], const
 
 struct FastPlan {
   int U, NT, RPU, NG, grid;
+  int HPT, QT;                 // query heads per row tile, row tiles per KV head
   long long total_runs, shift;
-  size_t off_partial, off_group, off_sync, sync_bytes, off_total;
+  size_t off_partial, off_group, off_sync, sync_bytes, off_parts, off_total;
 };
 
 // sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
 void make_plan(const Problem& P, int sms, FastPlan* pl) {
-  pl->U = P.L * P.Bt * P.Hkv;
+  const int G = P.Hq / P.Hkv;
+  pl->HPT = kRows / P.w < G ? kRows / P.w : G;
+  pl->QT = (G + pl->HPT - 1) / pl->HPT;
+  pl->U = P.L * P.Bt * P.Hkv * pl->QT;
   pl->NT = (int)((P.N + kTile - 1) / kTile);
   pl->RPU = (pl->NT + kRunTiles - 1) / kRunTiles;
   pl->NG = (pl->RPU + kGroupRuns - 1) / kGroupRuns;
@@ -966,6 +987,8 @@ void make_plan(const Problem& P, int sms, FastPlan* pl) {
   pl->off_sync = off;      // [U][NG] group counters, [U] unit counters, [U][128] log-sum-exp slots
   pl->sync_bytes = ((size_t)pl->U * pl->NG + (size_t)pl->U) * sizeof(int) + (size_t)pl->U * kRows * sizeof(float);
   off += align_up(pl->sync_bytes);
+  pl->off_parts = off;         // partial group aggregates [QT][L*Bt*Hkv][N], only with several row tiles
+  if (pl->QT > 1) off += align_up((size_t)pl->U * P.N * sizeof(float));
   pl->off_total = off;
 }
 
@@ -1005,12 +1028,11 @@ kvc_status launch_w(int W, const FastParams& fp, int grid, cudaStream_t st) {
 bool score_sm100_supported(const Problem& P) {
   if (P.dtype != KVC_BF16 || !P.contiguous_groups) return false;
   if (P.w != 8 && P.w != 16 && P.w != 32 && P.w != 64 && P.w != 128) return false;
-  const int G = P.Hq / P.Hkv;
-  if ((long long)G * P.w > kRows) return false;
-  if (P.L > kMaxFastLayers || (long long)P.L * P.Bt * P.Hkv > (1 << 24)) return false;
+  if (P.L > kMaxFastLayers) return false;
   if (P.N >= (1LL << 30)) return false;
   FastPlan pl;
   make_plan(P, 0, &pl);
+  if ((long long)P.L * P.Bt * P.Hkv * pl.QT > (1 << 24)) return false;
   if ((pl.total_runs + 4096) * kRunTiles + pl.shift >= (1LL << 31)) return false;   // 32-bit sequence indices
   return encode_fn() != nullptr;
 }
@@ -1024,7 +1046,8 @@ size_t score_sm100_workspace_bytes(const Problem& P) {
 // Returns KVC_ERR_UNSUPPORTED (without setting an error) when the tensor maps cannot be encoded
 // for these strides; the caller then uses the CUDA-core path.
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
-                              int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
+                              int* device_status, void* ws, size_t ws_bytes, cudaStream_t st,
+                              const float** parts_out, int* row_tiles_out) {
   const int sms = sm_count();
   if (sms < 1) return KVC_ERR_UNSUPPORTED;
   FastPlan pl;
@@ -1038,7 +1061,7 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
     const unsigned kb[4] = {64, (unsigned)kTile, 1, 1};
     const long long qd[4] = {P.d, P.w, P.Hq, P.Bt};
     const long long qs[3] = {P.qs[2] * 2, P.qs[1] * 2, P.qs[0] * 2};
-    const unsigned qb[4] = {64, (unsigned)P.w, (unsigned)G, 1};
+    const unsigned qb[4] = {64, (unsigned)P.w, (unsigned)pl.HPT, 1};
     if (!encode_map(&fp.k_maps[l], k.p[l], kd, ks, kb)) return KVC_ERR_UNSUPPORTED;
     if (!encode_map(&fp.q_maps[l], q.p[l], qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
   }
@@ -1052,15 +1075,20 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.unit_counter = fp.group_counter + (size_t)pl.U * pl.NG;
   fp.lse2 = reinterpret_cast<unsigned int*>(fp.unit_counter + pl.U);
   fp.status = device_status;
-  fp.scores = scores;
-  fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G; fp.R = G * P.w;
+  float* parts = pl.QT > 1 ? reinterpret_cast<float*>(w + pl.off_parts) : nullptr;
+  fp.scores = pl.QT > 1 ? parts : scores;
+  *parts_out = parts;
+  *row_tiles_out = pl.QT;
+  fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G;
+  fp.HPT = pl.HPT; fp.QT = pl.QT; fp.w = P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
   fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.NG = pl.NG; fp.grid = pl.grid;
   fp.total_runs = (unsigned int)pl.total_runs; fp.shift = (int)pl.shift;
   fp.step_u = pl.grid / pl.RPU; fp.step_j = pl.grid % pl.RPU;
-  fp.step_h = fp.step_u % P.Hkv;
-  fp.step_b = (fp.step_u / P.Hkv) % P.Bt;
-  fp.step_l = fp.step_u / P.Hkv / P.Bt;
+  fp.step_q = fp.step_u % pl.QT;
+  fp.step_h = (fp.step_u / pl.QT) % P.Hkv;
+  fp.step_b = (fp.step_u / pl.QT / P.Hkv) % P.Bt;
+  fp.step_l = fp.step_u / pl.QT / P.Hkv / P.Bt;
   fp.sl2e = P.scale * kLog2eF;
   fp.agg_group = P.agg_group;
   const bool mean = P.agg_task == KVC_AGG_MEAN;

@@ -148,6 +148,29 @@ def test_explicit_group_map_and_scale():
     check_all(wl, desc, cfg.budget)
 
 
+@pytest.mark.parametrize("Hq,Hkv,w,agg_task,agg_group,q_pos0", [
+    (8, 2, 64, 0, 0, None),     # 256 window rows per KV head: two row tiles of two query heads
+    (6, 2, 64, 0, 0, None),     # three query heads per KV head: the second row tile is short
+    (14, 2, 32, 0, 1, None),    # seven query heads, tiles of four and three, group max
+    (4, 1, 128, 1, 0, None),    # one query head per row tile, task mean
+    (8, 2, 64, 0, 0, 700),      # the causal window mask cuts through the context
+    (7, 1, 64, 1, 1, 1300),
+])
+def test_more_window_rows_than_one_accumulator_tile(Hq, Hkv, w, agg_task, agg_group, q_pos0):
+    """A GQA group whose window rows exceed 128 is scored in row tiles of whole query heads; the
+    group aggregate (Eq. 15) is then assembled from the tiles' parts."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("rowtiles", 2, Hq, Hkv, 128, 1500, w, dtype="bf16", retention=0.3,
+                           elem_std=1.0, hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    for augment in (1, 0):
+        kw = dict(agg_task=agg_task, agg_group=agg_group, augment_head_mean=augment)
+        if q_pos0 is not None:
+            kw["q_pos0"] = q_pos0
+        desc = kvc.desc_from_config(cfg, **kw)
+        check_all(wl, desc, cfg.budget)
+
+
 def test_batch_and_strided_inputs():
     """Two sequences; K/V/Q are views into larger buffers (non-dense batch/head/token strides)."""
     dev = _cuda()
