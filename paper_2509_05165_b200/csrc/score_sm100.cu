@@ -6,15 +6,23 @@
 //                        accumulator in TMEM.  Query rows sit on TMEM lanes, so the softmax
 //                        denominator of a row (Eq. 3) is an in-thread sum: every row keeps a
 //                        reference exponent and a running sum of 2^(logit - reference).
-//   exchange             a run of kRunTiles consecutive tiles of one (layer, sequence, KV head)
-//                        unit yields one record of (reference, sum) per row, which the pass-1
-//                        epilogue writes to global memory and counts into its group of
-//                        kGroupRuns runs.  Every group and every unit has a fixed folding CTA
-//                        (round-robin): its exchange warp waits for the count, folds the group's
-//                        records (fixed order) into one and counts the group into the unit, or
-//                        folds a unit's group records into the rows' log-sum-exp.  Each fold is
-//                        one batch of loads, the folds are spread evenly over the CTAs, and none
-//                        of it sits on the path of the CTA's own tiles.
+//   exchange             a run of RT consecutive tiles of one (layer, sequence, KV head) unit
+//                        yields one (reference, sum) per row.  The short way: every row has a
+//                        fixed reference (its logit against token 0, from a small kernel that
+//                        runs first) and one 64-bit word; the pass-1 epilogue rescales the run's
+//                        sum to that reference, converts it to fixed point (2^-20) and adds it,
+//                        together with an arrival count in the top byte, with one integer
+//                        reduction.  Integer addition makes the total independent of the order
+//                        of arrival, and sum and count travel in one word, so a reader needs no
+//                        fence: the word is complete when its count equals the unit's runs.
+//                        That is two round trips to L2 between the last pass-1 tile of a unit
+//                        and its first pass-2 tile.  The long way, always taken as well: the
+//                        run's record of (reference, sum) per row goes to global memory and is
+//                        counted into its group of kGroupRuns runs; every group and every unit
+//                        has a fixed folding CTA (round-robin) whose exchange warp waits for the
+//                        count and folds in a fixed order, down to the rows' log-sum-exp.  Pass 2
+//                        uses it for the rows whose word says that some run's sum did not fit
+//                        the fixed-point range (a token about 14 nats above token 0).
 //   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
 //                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
 //                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
@@ -28,7 +36,8 @@
 // aggregates that the Eq. 16 kernel combines in a fixed order.
 //
 // Every CTA walks one static sequence that alternates a pass-1 tile with a pass-2 tile; the
-// pass-2 stream trails the pass-1 stream by `shift` tiles.  A pass-2 tile only ever waits for
+// pass-2 stream trails the pass-1 stream by `shift` tiles (two runs where a unit has no more
+// runs than there are CTAs: 38 MB of K at 148 CTAs, which L2 still holds).  A pass-2 tile only ever waits for
 // pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot deadlock while all
 // CTAs are resident.  Every wait (mbarrier or global flag) is bounded; on expiry the kernel
 // records KVC_ERR_TIMEOUT, stops computing and drains.
@@ -44,10 +53,10 @@
 #include "kvc_internal.cuh"
 
 #ifndef KVC_SCORE_RUN_TILES
-#define KVC_SCORE_RUN_TILES 8      // tiles per run
+#define KVC_SCORE_RUN_TILES 4      // tiles per run
 #endif
-#ifndef KVC_SCORE_LAG_EXTRA
-#define KVC_SCORE_LAG_EXTRA 2      // runs of slack between a unit's last pass-1 run and its first pass-2 run
+#ifndef KVC_SCORE_LAG_TILES
+#define KVC_SCORE_LAG_TILES 0      // tiles of slack beyond the runs a unit's statistics have to wait for
 #endif
 #ifndef KVC_SCORE_PREFETCH
 #define KVC_SCORE_PREFETCH 2       // pass-1 tiles prefetched into L2 ahead of their load
@@ -74,7 +83,7 @@ namespace {
 constexpr int kTile = 128;            // tokens per tile = MMA M = MMA N
 constexpr int kFastThreads = 512;
 constexpr int kRows = 128;            // query rows per unit handled by one MMA (R <= 128)
-constexpr int kRunTiles = KVC_SCORE_RUN_TILES;
+constexpr int kMinRunTiles = KVC_SCORE_RUN_TILES;   // runs are longer only where a unit would otherwise have more than 255
 constexpr int kGroupRuns = 8;         // runs whose partials are folded together at the first level
 constexpr int kQSlots = 3;
 constexpr int kPrefetch = KVC_SCORE_PREFETCH;
@@ -92,12 +101,16 @@ struct FastParams {
   int* group_counter;          // [U][NG], preset to -1
   int* unit_counter;           // [U], preset to -1
   unsigned int* lse2;          // [U][128] fp32 bits, preset to 0xffffffff ("not there yet")
+  unsigned long long* acc;     // [U][128], preset to 0: per row  arrivals << 56 | overflows << 48 | sum in units
+                               // of 2^-20 of 2^(logit - ref[row]), added to by every run of the unit
+  const float* ref;            // [U][128]: the row's reference exponent (its scaled logit against token 0)
   int* status;                 // device status word (may be null)
   float* scores;               // [L*Bt*Hkv][N], or with QT > 1 the partial aggregates [QT][L*Bt*Hkv][N]
   int L, Bt, Hkv, G;
   int HPT, QT, w;              // query heads per row tile, row tiles per KV head, window rows per query head
   long long N, q_pos0;
   int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
+  int RT;                      // tiles per run
   int step_u, step_j;          // grid = step_u * RPU + step_j: how a CTA's next run moves (unit, run in unit)
   int step_l, step_b, step_h, step_q;  // step_u = ((step_l * Bt + step_b) * Hkv + step_h) * QT + step_q
   unsigned int total_runs;     // U * RPU
@@ -244,6 +257,19 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const unsigned int* p) {
 __device__ __forceinline__ void st_relaxed_u32(unsigned int* p, uint32_t v) {
   asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ float lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void red_add_release(int* p, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -281,7 +307,7 @@ __device__ __forceinline__ void combine(float& M, float& Ls, float m, float l) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// The static per-CTA sequence.  Stream position idx -> (run ordinal, tile); a run is kRunTiles
+// The static per-CTA sequence.  Stream position idx -> (run ordinal, tile); a run is RT
 // consecutive tiles of one unit, runs are dealt to the CTAs round-robin.
 // ------------------------------------------------------------------------------------------------
 // Walks one stream of this CTA: position -> (run, tile).  Run k of the CTA is the global run
@@ -289,7 +315,7 @@ __device__ __forceinline__ void combine(float& M, float& Ls, float m, float l) {
 // increments come from the host), because a division would queue behind the exponentials in the
 // special-function pipe.
 struct Cursor {
-  int t;            // position inside the run, 0 .. kRunTiles-1
+  int t;            // position inside the run, 0 .. RT-1
   int u, j;         // unit, run inside the unit
   int l, b, h, q;   // the unit's layer, sequence, KV head, row tile
   __device__ __forceinline__ void init(const FastParams& P) {
@@ -307,10 +333,10 @@ struct Cursor {
   __device__ __forceinline__ int rows(const FastParams& P) const { return min(P.HPT, P.G - q * P.HPT) * P.w; }
   // index of the (layer, sequence, KV head)
   __device__ __forceinline__ int kv_unit(const FastParams& P) const { return (l * P.Bt + b) * P.Hkv + h; }
-  __device__ __forceinline__ int tile() const { return j * kRunTiles + t; }
-  __device__ __forceinline__ bool valid(const FastParams& P) const { return tile() < P.NT; }
+  __device__ __forceinline__ int tile(const FastParams& P) const { return j * P.RT + t; }
+  __device__ __forceinline__ bool valid(const FastParams& P) const { return tile(P) < P.NT; }
   // last valid tile of its run
-  __device__ __forceinline__ bool last(const FastParams& P) const { return t == kRunTiles - 1 || tile() + 1 >= P.NT; }
+  __device__ __forceinline__ bool last(const FastParams& P) const { return t == P.RT - 1 || tile(P) + 1 >= P.NT; }
   __device__ __forceinline__ void next_run(const FastParams& P) {
     j += P.step_j;
     int c = 0;
@@ -325,7 +351,7 @@ struct Cursor {
     l += P.step_l + c;
   }
   __device__ __forceinline__ void advance(const FastParams& P) {
-    if (++t == kRunTiles) { t = 0; next_run(P); }
+    if (++t == P.RT) { t = 0; next_run(P); }
   }
 };
 
@@ -358,6 +384,28 @@ struct SmemLayout {
   static constexpr int kTotal = kStats + kRows * 8;
   static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
+
+// The pushed statistics of one row (see FastParams::acc).
+constexpr int kAccFracBits = 20;                              // the sum counts units of 2^-20
+constexpr float kAccLimitLog2 = 20.f;                         // a run's contribution must stay below 2^20
+constexpr unsigned long long kAccArrival = 1ull << 56, kAccOverflow = 1ull << 48;
+constexpr unsigned long long kAccSumMask = kAccOverflow - 1;
+
+// Bounded poll of a row's pushed statistics until all `runs` runs of the unit have arrived.
+__device__ __noinline__ unsigned long long poll_acc_slow(const unsigned long long* src, unsigned int runs,
+                                                         volatile int* abort_word) {
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  unsigned long long v;
+  while ((unsigned int)((v = ld_relaxed_u64(src)) >> 56) != runs) {
+    __nanosleep(100);
+    if ((++spins & 255u) == 0) {
+      if (*abort_word) break;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
+    }
+  }
+  return v;
+}
 
 // Bounded poll of a log-sum-exp slot (the value itself is the flag).
 __device__ __noinline__ uint32_t poll_lse_slow(const unsigned int* src, volatile int* abort_word) {
@@ -491,7 +539,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   // this CTA's share of the runs and the length of its sequence
   // (the host keeps all of these below 2^31)
   const int my_runs = (P.total_runs > blockIdx.x) ? (int)((P.total_runs - blockIdx.x + P.grid - 1) / P.grid) : 0;
-  const int my_tiles = my_runs * kRunTiles;                  // stream length (some positions hold no tile)
+  const int my_tiles = my_runs * P.RT;                  // stream length (some positions hold no tile)
   const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
   const uint32_t q_bytes = (uint32_t)(P.HPT * P.w) * D * 2;   // the whole box arrives (rows outside the tensor as zeros)
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
@@ -513,7 +561,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         if (ahead_pos >= my_tiles) return;
         if (ahead.valid(P)) {
           for (int hf = 0; hf < SL::kHalves; ++hf)
-            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile() * kTile, ahead.h, ahead.b);
+            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile(P) * kTile, ahead.h, ahead.b);
         }
         ahead.advance(P);
         ++ahead_pos;
@@ -543,7 +591,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
               // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
               for (int hf = 0; hf < SL::kHalves; ++hf)
                 tma_load_4d(sbase + SL::kK + kr.i * SL::kTileBytes + hf * (kTile * 128), P.k_maps + c.l,
-                            bar_kfull(kr.i), hf * 64, c.tile() * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
+                            bar_kfull(kr.i), hf * 64, c.tile(P) * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
               kr.next(SL::kStages);
               if (nk < SL::kStages) ++nk;
             }
@@ -727,6 +775,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     int n1 = 0;
     KVC_TR_DECL(e_t = 0, e_c = 0, e_b = 0, e_s = KVC_TR_NOW());
     float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
+    float row_ref = 0.f;                              // the row's reference exponent for the pushed sum
     bool ok = true;
 
     // 32 unmasked logits against the row's current reference: no maximum, packed arithmetic.
@@ -762,9 +811,10 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     c.init(P);
     for (int idx = 0; idx < my_tiles; ++idx, c.advance(P)) {
       if (!c.valid(P)) continue;
-      const int tile = c.tile();
+      const int tile = c.tile(P);
       const bool run_ends = c.last(P);
       const bool row_used = row < c.rows(P);
+      if (c.t == 0 && half == 0) row_ref = __ldg(P.ref + (long long)c.u * kRows + row);   // used at the run's end
       const int buf = n1 & 1;
       KVC_TR(e_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word));
       tc_fence_after();
@@ -801,6 +851,17 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           float M = row_used ? mref : -INFINITY, Ls = row_used ? lsum : 0.f;
           combine(M, Ls, other.x, other.y);
           reinterpret_cast<float2*>(P.partial)[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
+          {
+            // the short way: add the run's sum, rescaled to the row's fixed reference, to the
+            // row's 64-bit word (integer addition: the total does not depend on the order)
+            unsigned long long add = kAccArrival;
+            if (Ls > 0.f) {
+              const float lv = lg2(Ls) + (M - row_ref);                 // log2 of the contribution
+              if (lv < kAccLimitLog2) add += __float2ull_rn(ex2(lv + (float)kAccFracBits));
+              else add += kAccOverflow;                                  // the rows' records decide instead
+            }
+            red_add_u64(P.acc + (long long)c.u * kRows + row, add);
+          }
           __syncwarp();
           if (lane == 0) {
             // the four warps order their parts of the record through this counter (release /
@@ -827,25 +888,62 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 
     Cursor cu;
     cu.init(P);
+    unsigned long long early_word = 0ull;             // a coming run's pushed word and reference, fetched ahead
+    float early_ref = 0.f;
+    int early_u = -1;                                 // ... and the unit they belong to
+    int lse_u = -1, lse_j = -1;                       // the run whose values this warpgroup holds
+    if (my_tiles > 0) {
+      early_word = ld_relaxed_u64(P.acc + (long long)cu.u * kRows + trow);
+      early_ref = __ldg(P.ref + (long long)cu.u * kRows + trow);
+      early_u = cu.u;
+    }
     for (int idx = 0; idx < my_tiles; ++idx, cu.advance(P)) {
       if (!cu.valid(P)) continue;
-      const int tile = cu.tile();
+      const int tile = cu.tile(P);
       const int rows_u = cu.rows(P);
       const int n_chunks = (rows_u + 31) / 32;
-      if (cu.t == 0) {
-        // a new run: wait for its unit's log-sum-exp (the value itself is the flag)
-        uint32_t bits = 0xffffffffu;
+      if (cu.u != lse_u || cu.j != lse_j) {
+        lse_u = cu.u; lse_j = cu.j;
+        // a new run: its unit's log-sum-exp.  The short way: the row's pushed word, complete once
+        // every run of the unit has arrived (fetched a tile or two ago; polled if it was not
+        // complete then).  If a run's sum did not fit, or the word is not in use, the folded
+        // records decide (the value is its own flag).
+        float lse = 0.f;
         KVC_TR_DECL(f_l0 = KVC_TR_NOW());
         if (ok && trow < rows_u) {
-          const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
-          bits = ld_relaxed_u32(src);
-          if (bits == 0xffffffffu) bits = poll_lse_slow(src, abort_word);
+          bool pushed = false;
+          {
+            if (early_u != cu.u) { early_word = 0ull; early_ref = __ldg(P.ref + (long long)cu.u * kRows + trow); }
+            unsigned long long word = early_word;
+            if ((unsigned int)(word >> 56) != (unsigned int)P.RPU)
+              word = poll_acc_slow(P.acc + (long long)cu.u * kRows + trow, (unsigned int)P.RPU, abort_word);
+            const unsigned long long sum = word & kAccSumMask;
+            if (((word >> 48) & 0xffull) == 0 && sum != 0) {
+              lse = early_ref + lg2((float)sum) - (float)kAccFracBits;
+              pushed = true;
+            }
+          }
+          if (!pushed) {
+            const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
+            uint32_t bits = ld_relaxed_u32(src);
+            if (bits == 0xffffffffu) bits = poll_lse_slow(src, abort_word);
+            lse = __uint_as_float(bits);
+          }
         }
+        early_u = -1;
         named_bar(1, 128);                             // everyone is done with the previous unit's values
-        neg_lse[trow] = (trow < rows_u) ? -__uint_as_float(bits) : 0.f;
+        neg_lse[trow] = (trow < rows_u) ? -lse : 0.f;
         named_bar(1, 128);
         KVC_TR_SINCE(f_l, f_l0);
         if (*abort_word) ok = false;
+      }
+      if (early_u < 0 && cu.t >= P.RT - 2 && idx + (P.RT - cu.t) < my_tiles) {
+        // the next run's word and reference: in flight while the rest of this run is computed
+        Cursor nx = cu;
+        nx.next_run(P);
+        early_word = ld_relaxed_u64(P.acc + (long long)nx.u * kRows + trow);
+        early_ref = __ldg(P.ref + (long long)nx.u * kRows + trow);
+        early_u = nx.u;
       }
       const int buf = 2 + (n2 & 1);
       const uint32_t tmem_col = (uint32_t)buf * kTile;
@@ -926,6 +1024,36 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// The rows' reference exponents: the scaled logit (base 2) of every window row against token 0 of
+// its KV head, which every row sees.  Only a common scale for the pushed sums: a row's sum of
+// 2^(logit - ref) is then at least about 1, so fixed point with 20 fractional bits keeps it.
+// ------------------------------------------------------------------------------------------------
+struct RefParams {
+  int Bt, Hkv, G, HPT, QT, w, d;
+  long long qs0, qs1, qs2, kvs0, kvs1;
+  float sl2e;
+};
+
+__global__ void __launch_bounds__(kRows)
+score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ ref) {
+  const int u = blockIdx.x, row = threadIdx.x;
+  const int uh = u / P.QT, qt = u - uh * P.QT;
+  const int lb = uh / P.Hkv, h = uh - lb * P.Hkv;
+  const int l = lb / P.Bt, b = lb - l * P.Bt;
+  const int rows_u = min(P.HPT, P.G - qt * P.HPT) * P.w;
+  float r = 0.f;
+  if (row < rows_u) {
+    const int j = h * P.G + qt * P.HPT + row / P.w, m = row % P.w;
+    const __nv_bfloat16* qv = reinterpret_cast<const __nv_bfloat16*>(qp.p[l]) + b * P.qs0 + j * P.qs1 + m * P.qs2;
+    const __nv_bfloat16* kv = reinterpret_cast<const __nv_bfloat16*>(kp.p[l]) + b * P.kvs0 + h * P.kvs1;
+    float acc = 0.f;
+    for (int t = 0; t < P.d; ++t) acc = fmaf(__bfloat162float(qv[t]), __bfloat162float(kv[t]), acc);
+    r = acc * P.sl2e;
+  }
+  ref[(long long)u * kRows + row] = r;
+}
+
+// ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -959,10 +1087,10 @@ bool encode_map(CUtensorMap* m, const void* base, const long long dims[4], const
 }
 
 struct FastPlan {
-  int U, NT, RPU, NG, grid;
+  int U, NT, RPU, NG, grid, RT;
   int HPT, QT;                 // query heads per row tile, row tiles per KV head
   long long total_runs, shift;
-  size_t off_partial, off_group, off_sync, sync_bytes, off_parts, off_total;
+  size_t off_partial, off_group, off_sync, sync_bytes, off_parts, off_acc, off_ref, off_total;
 };
 
 // sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
@@ -972,21 +1100,25 @@ void make_plan(const Problem& P, int sms, FastPlan* pl) {
   pl->QT = (G + pl->HPT - 1) / pl->HPT;
   pl->U = P.L * P.Bt * P.Hkv * pl->QT;
   pl->NT = (int)((P.N + kTile - 1) / kTile);
-  pl->RPU = (pl->NT + kRunTiles - 1) / kRunTiles;
+  pl->RT = kMinRunTiles;
+  if ((pl->NT + pl->RT - 1) / pl->RT > 255) pl->RT = (pl->NT + 254) / 255;   // the arrivals of a unit are counted in 8 bits
+  pl->RPU = (pl->NT + pl->RT - 1) / pl->RT;
   pl->NG = (pl->RPU + kGroupRuns - 1) / kGroupRuns;
   pl->total_runs = (long long)pl->U * pl->RPU;
   pl->grid = sms > 0 ? (int)(pl->total_runs < sms ? pl->total_runs : sms) : 1;
-  // pass 2 of a run starts once every CTA has been through the rest of the run's unit (at most
-  // ceil(RPU / grid) runs later) plus some runs that hide the exchange; half a run staggers the
-  // two streams so that they change runs (and Q tiles) at different moments
-  const long long lag_runs = (pl->RPU + pl->grid - 1) / pl->grid + KVC_SCORE_LAG_EXTRA;
-  pl->shift = lag_runs * kRunTiles + kRunTiles / 2;
+  // pass 2 of a run starts once every CTA has been through the rest of the run's unit, at most
+  // ceil(RPU / grid) runs later, and through one run more, which covers the exchange (the pushed
+  // sums take two round trips to L2); the K rows of that many tiles are still in L2 then
+  const long long lag_runs = (pl->RPU + pl->grid - 1) / pl->grid + 1;
+  pl->shift = lag_runs * pl->RT + KVC_SCORE_LAG_TILES;
   size_t off = 0;
   pl->off_partial = off; off += align_up((size_t)pl->total_runs * 64 * sizeof(float4));
   pl->off_group = off; off += align_up((size_t)pl->U * pl->NG * 64 * sizeof(float4));
   pl->off_sync = off;      // [U][NG] group counters, [U] unit counters, [U][128] log-sum-exp slots
   pl->sync_bytes = ((size_t)pl->U * pl->NG + (size_t)pl->U) * sizeof(int) + (size_t)pl->U * kRows * sizeof(float);
   off += align_up(pl->sync_bytes);
+  pl->off_acc = off; off += align_up((size_t)pl->U * kRows * sizeof(unsigned long long));
+  pl->off_ref = off; off += align_up((size_t)pl->U * kRows * sizeof(float));
   pl->off_parts = off;         // partial group aggregates [QT][L*Bt*Hkv][N], only with several row tiles
   if (pl->QT > 1) off += align_up((size_t)pl->U * P.N * sizeof(float));
   pl->off_total = off;
@@ -1033,7 +1165,7 @@ bool score_sm100_supported(const Problem& P) {
   FastPlan pl;
   make_plan(P, 0, &pl);
   if ((long long)P.L * P.Bt * P.Hkv * pl.QT > (1 << 24)) return false;
-  if ((pl.total_runs + 4096) * kRunTiles + pl.shift >= (1LL << 31)) return false;   // 32-bit sequence indices
+  if ((pl.total_runs + 4096) * pl.RT + pl.shift >= (1LL << 31)) return false;   // 32-bit sequence indices
   return encode_fn() != nullptr;
 }
 
@@ -1074,6 +1206,18 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.group_counter = reinterpret_cast<int*>(w + pl.off_sync);
   fp.unit_counter = fp.group_counter + (size_t)pl.U * pl.NG;
   fp.lse2 = reinterpret_cast<unsigned int*>(fp.unit_counter + pl.U);
+  fp.acc = reinterpret_cast<unsigned long long*>(w + pl.off_acc);
+  float* ref = reinterpret_cast<float*>(w + pl.off_ref);
+  fp.ref = ref;
+  {
+    KVC_CUDA(cudaMemsetAsync(fp.acc, 0, (size_t)pl.U * kRows * sizeof(unsigned long long), st));
+    RefParams rp;
+    rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.w = P.w; rp.d = P.d;
+    rp.qs0 = P.qs[0]; rp.qs1 = P.qs[1]; rp.qs2 = P.qs[2]; rp.kvs0 = P.kvs[0]; rp.kvs1 = P.kvs[1];
+    rp.sl2e = P.scale * kLog2eF;
+    score_ref_kernel<<<pl.U, kRows, 0, st>>>(rp, q, k, ref);
+    KVC_LAUNCH_CHECK("score_ref_kernel");
+  }
   fp.status = device_status;
   float* parts = pl.QT > 1 ? reinterpret_cast<float*>(w + pl.off_parts) : nullptr;
   fp.scores = pl.QT > 1 ? parts : scores;
@@ -1082,7 +1226,7 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G;
   fp.HPT = pl.HPT; fp.QT = pl.QT; fp.w = P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
-  fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.NG = pl.NG; fp.grid = pl.grid;
+  fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.RT = pl.RT; fp.NG = pl.NG; fp.grid = pl.grid;
   fp.total_runs = (unsigned int)pl.total_runs; fp.shift = (int)pl.shift;
   fp.step_u = pl.grid / pl.RPU; fp.step_j = pl.grid % pl.RPU;
   fp.step_q = fp.step_u % pl.QT;

@@ -171,6 +171,19 @@ def test_more_window_rows_than_one_accumulator_tile(Hq, Hkv, w, agg_task, agg_gr
         check_all(wl, desc, cfg.budget)
 
 
+@pytest.mark.parametrize("scale", [2.0, 0.5])
+def test_logits_far_above_the_first_tokens(scale):
+    """A large logit scale: for most window rows some token lies tens of nats above token 0, whose
+    logit is the reference of the rows' pushed fixed-point sums, so those rows' statistics have to
+    come from the folded (reference, sum) records instead; other rows still take the short way."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("steep", 2, 8, 2, 128, 1500, 32, dtype="bf16", retention=0.3, elem_std=1.0,
+                           hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    desc = kvc.desc_from_config(cfg, scale=scale)
+    check_all(wl, desc, cfg.budget, check_e2e=False)
+
+
 def test_batch_and_strided_inputs():
     """Two sequences; K/V/Q are views into larger buffers (non-dense batch/head/token strides)."""
     dev = _cuda()
