@@ -1046,8 +1046,21 @@ score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ re
     const int j = h * P.G + qt * P.HPT + row / P.w, m = row % P.w;
     const __nv_bfloat16* qv = reinterpret_cast<const __nv_bfloat16*>(qp.p[l]) + b * P.qs0 + j * P.qs1 + m * P.qs2;
     const __nv_bfloat16* kv = reinterpret_cast<const __nv_bfloat16*>(kp.p[l]) + b * P.kvs0 + h * P.kvs1;
+    // 16-byte pieces (rows are 16-byte aligned), all in flight at once; products added in order
+    const uint4* q4 = reinterpret_cast<const uint4*>(qv);
+    const uint4* k4 = reinterpret_cast<const uint4*>(kv);
     float acc = 0.f;
-    for (int t = 0; t < P.d; ++t) acc = fmaf(__bfloat162float(qv[t]), __bfloat162float(kv[t]), acc);
+#pragma unroll 4
+    for (int t = 0; t < P.d / 8; ++t) {
+      const uint4 a = __ldg(q4 + t), b2 = __ldg(k4 + t);
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b2.x, b2.y, b2.z, b2.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        // a bf16 is the upper half of the fp32 with the same value
+        acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
+        acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
+      }
+    }
     r = acc * P.sl2e;
   }
   ref[(long long)u * kRows + row] = r;
