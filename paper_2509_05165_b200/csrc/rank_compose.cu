@@ -69,13 +69,29 @@ sort_count_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* id
   const int shift = 8 * pass;
   for (int i = tid; i < kRadix; i += kSortThreads) hist[i] = 0;
   __syncthreads();
+  // counting does not care about the order inside the tile: where the segment allows 16-byte
+  // loads, a thread takes 8 consecutive elements with two of them
   const long long w0 = (long long)tile * kTileItems + (long long)warp * kWarpItems;
+  const uint32_t* base = pass == 0 ? reinterpret_cast<const uint32_t*>(s_in) : io.src_k;
+  const bool wide = (reinterpret_cast<uintptr_t>(base) & 15u) == 0 && w0 + kWarpItems <= N;
+  uint32_t keys[kItems];
+  if (wide) {
+    const uint4* src = reinterpret_cast<const uint4*>(base) + (w0 >> 2) + lane * 2;
+    const uint4 a = src[0], b = src[1];
+    keys[0] = a.x; keys[1] = a.y; keys[2] = a.z; keys[3] = a.w;
+    keys[4] = b.x; keys[5] = b.y; keys[6] = b.z; keys[7] = b.w;
+    if (pass == 0) {
+#pragma unroll
+      for (int k = 0; k < kItems; ++k) keys[k] = score_to_key(__uint_as_float(keys[k]));
+    }
+  }
 #pragma unroll
   for (int k = 0; k < kItems; ++k) {
     const long long i = w0 + k * 32 + lane;
-    const bool valid = i < N;
+    const bool valid = wide || i < N;
     uint32_t key = 0;
-    if (valid) key = (pass == 0) ? score_to_key(s_in[i]) : io.src_k[i];
+    if (wide) key = keys[k];
+    else if (valid) key = (pass == 0) ? score_to_key(s_in[i]) : io.src_k[i];
     const uint32_t digit = (key >> shift) & 0xffu;
     if (pass < 3) {
       // the low digits are spread over their 256 bins: plain shared-memory atomics hardly collide
