@@ -171,6 +171,25 @@ def test_more_window_rows_than_one_accumulator_tile(Hq, Hkv, w, agg_task, agg_gr
         check_all(wl, desc, cfg.budget)
 
 
+@pytest.mark.parametrize("Hq,Hkv,w,d,N,batch,q_pos0", [
+    (4, 4, 32, 128, 1000, 1, None),      # no grouping: one query head per KV head
+    (8, 2, 8, 64, 2100, 2, None),        # short window, two sequences, head size 64
+    (16, 2, 16, 128, 900, 1, None),      # eight query heads of 16 rows fill the accumulator exactly
+    (8, 8, 128, 128, 600, 1, None),      # one query head of 128 rows per KV head
+    (8, 2, 32, 128, 1300, 1, 5000),      # task-aware: the window lies after the context, nothing is masked
+    (8, 2, 32, 128, 4096 + 64, 1, None), # enough runs per unit for several groups of folded records
+])
+def test_tensor_core_path_shapes(Hq, Hkv, w, d, N, batch, q_pos0):
+    """bf16 shapes of the tensor-core scoring path: group sizes, window lengths, head sizes, batch."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("shapes", 2, Hq, Hkv, d, N, w, batch=batch, dtype="bf16", retention=0.3,
+                           elem_std=1.0, hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    kw = {} if q_pos0 is None else {"q_pos0": q_pos0}
+    desc = kvc.desc_from_config(cfg, **kw)
+    check_all(wl, desc, cfg.budget)
+
+
 @pytest.mark.parametrize("scale", [2.0, 0.5])
 def test_logits_far_above_the_first_tokens(scale):
     """A large logit scale: for most window rows some token lies tens of nats above token 0, whose
