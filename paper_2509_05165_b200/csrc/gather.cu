@@ -3,7 +3,8 @@
 //
 // Pure data movement: every output row is one contiguous head_dim-wide row of the cache.  A row
 // is moved by row_bytes / 16 lanes with one 16-byte load and one 16-byte store each; a warp
-// carries 32 / lanes_per_row rows of K and of V per step and several steps are kept in flight.
+// carries 32 / lanes_per_row rows of K and of V per step; parallelism comes from many resident
+// CTAs rather than from several rows per thread.
 // The per-layer counts and offsets are read on the device, so no host synchronisation is needed
 // between allocation and compaction.
 #include "kvc_internal.cuh"
@@ -12,7 +13,7 @@ namespace kvc {
 namespace {
 
 constexpr int kGatherThreads = 256;
-constexpr int kUnroll = 4;
+constexpr int kUnroll = 1;            // rows per thread and step: more of them in flight was slower (measured 1 to 8)
 
 struct GatherParams {
   int L, Bt, Hkv;
@@ -101,7 +102,7 @@ kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& 
   gp.rows_per_seq = budget * P.Hkv;
   const long long rows_per_block = kGatherThreads / gp.lanes_per_row;
   long long blocks = (gp.rows_per_seq + rows_per_block * kUnroll - 1) / (rows_per_block * kUnroll);
-  const long long cap = 148LL * 8 * 4;
+  const long long cap = 148LL * 128;   // measured best among 8 to 256 CTAs per SM's worth of grid
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   gather_kernel<<<dim3((unsigned)blocks, P.Bt), kGatherThreads, 0, st>>>(
