@@ -891,7 +891,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     unsigned long long early_word = 0ull;             // a coming run's pushed word and reference, fetched ahead
     float early_ref = 0.f;
     int early_u = -1;                                 // ... and the unit they belong to
-    int lse_u = -1, lse_j = -1;                       // the run whose values this warpgroup holds
     if (my_tiles > 0) {
       early_word = ld_relaxed_u64(P.acc + (long long)cu.u * kRows + trow);
       early_ref = __ldg(P.ref + (long long)cu.u * kRows + trow);
@@ -902,11 +901,10 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       const int tile = cu.tile(P);
       const int rows_u = cu.rows(P);
       const int n_chunks = (rows_u + 31) / 32;
-      if (cu.u != lse_u || cu.j != lse_j) {
-        lse_u = cu.u; lse_j = cu.j;
+      if (cu.t == 0) {
         // a new run: its unit's log-sum-exp.  The short way: the row's pushed word, complete once
         // every run of the unit has arrived (fetched a tile or two ago; polled if it was not
-        // complete then).  If a run's sum did not fit, or the word is not in use, the folded
+        // complete then).  If a run's sum did not fit, the folded
         // records decide (the value is its own flag).
         float lse = 0.f;
         KVC_TR_DECL(f_l0 = KVC_TR_NOW());
