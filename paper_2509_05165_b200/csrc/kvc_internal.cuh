@@ -67,7 +67,7 @@ size_t score_workspace_bytes(const Problem& P);
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
                         float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
 // The two implementations behind it: CUDA cores (any supported shape) and tcgen05 (bf16,
-// contiguous GQA groups, window of 8, 16, 32, 64 or 128 rows).
+// contiguous GQA groups, window of at most 128 rows).
 size_t score_generic_workspace_bytes(const Problem& P);
 kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
                                 const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,

@@ -32,7 +32,8 @@
 //
 // A unit is a (layer, sequence, KV head, row tile): the G x w window rows of a KV head are cut
 // into row tiles of at most 128 rows (whole query heads), so that any GQA group / window size
-// with w <= 128 runs here; with more than one row tile the pass-2 results are partial group
+// with w <= 128 runs here (w = 8, 16, 32, 64, 128 as compile-time specialisations, any other
+// length through one variant that reads it at run time); with more than one row tile the pass-2 results are partial group
 // aggregates that the Eq. 16 kernel combines in a fixed order.
 //
 // Every CTA walks one static sequence that alternates a pass-1 tile with a pass-2 tile; the
@@ -464,12 +465,14 @@ __device__ __noinline__ void p1_masked_half(uint32_t taddr, long long c_first, l
 }
 
 // Pass 2, one token (this thread's TMEM lane) against all query rows, any aggregator, with
-// masking.  Returns the group aggregate before the division of the mean.
+// masking.  Returns the group aggregate before the division of the mean.  W is the window length
+// where it is one of the specialised powers of two, 0 where it is only known at run time (`w`).
 template <int W, bool kTaskMean>
 __device__ __noinline__ float p2_generic_tile(uint32_t taddr, const float* neg_lse, int n_chunks, int R, float sl2e,
-                                              bool full, long long m_min, int agg_group) {
+                                              bool full, long long m_min, int agg_group, int w) {
   float gacc = (agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
   float hacc = kTaskMean ? 0.f : -INFINITY;
+  int m = 0;                                                             // row inside its query head (W == 0)
 #pragma unroll 1
   for (int j = 0; j < n_chunks; ++j) {
     uint32_t r[32];
@@ -479,11 +482,20 @@ __device__ __noinline__ float p2_generic_tile(uint32_t taddr, const float* neg_l
     for (int i = 0; i < 32; ++i) {
       const int col = j * 32 + i;
       float xi = fmaf(__uint_as_float(r[i]), sl2e, neg_lse[col]);       // log2 of the attention weight
-      if (!full && (col % W) < m_min) xi = -INFINITY;
+      bool head_done;
+      if (W > 0) {
+        constexpr int Wd = W > 0 ? W : 1;
+        if (!full && (col % Wd) < m_min) xi = -INFINITY;
+        head_done = (col + 1) % Wd == 0;
+      } else {
+        if (!full && m < m_min) xi = -INFINITY;
+        head_done = ++m == w;
+        if (head_done) m = 0;
+      }
       if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
-      if ((col + 1) % W == 0) {                                          // a query head is complete
+      if (head_done) {                                                   // a query head is complete
         if (col < R) {
-          const float s_task = kTaskMean ? hacc * (1.0f / W) : ex2(hacc);
+          const float s_task = kTaskMean ? hacc / (float)w : ex2(hacc);
           gacc = (agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
         }
         hacc = kTaskMean ? 0.f : -INFINITY;
@@ -769,7 +781,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const int row = quarter * 32 + lane;              // TMEM lane = query row
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + row;
-    const long long row_vis = min(P.N - 1, P.q_pos0 + (row % W));     // last key this row sees
+    const long long row_vis = min(P.N - 1, P.q_pos0 + (row % (W > 0 ? W : P.w)));     // last key this row sees
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
 
     int n1 = 0;
@@ -989,7 +1001,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           for (int i = 2; i < 30; i += 4) { a = max3(a, x[i], x[i + 1]); b = max3(b, x[i + 2], x[i + 3]); }
           hacc = max3(hacc, a, b);
           hacc = max3(hacc, x[30], x[31]);
-          if (((j + 1) * 32) % W == 0) {
+          if (((j + 1) * 32) % (W > 0 ? W : 1) == 0) {
             const float s_task = ex2(hacc);
             gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
             hacc = -INFINITY;
@@ -997,7 +1009,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         }
       } else {
         gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
-                                             c - P.q_pos0, P.agg_group);
+                                             c - P.q_pos0, P.agg_group, P.w);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(buf));
@@ -1162,7 +1174,8 @@ kvc_status launch_w(int W, const FastParams& fp, int grid, cudaStream_t st) {
     case 16: return launch_t<D, 16, M>(fp, grid, st);
     case 32: return launch_t<D, 32, M>(fp, grid, st);
     case 64: return launch_t<D, 64, M>(fp, grid, st);
-    default: return launch_t<D, 128, M>(fp, grid, st);
+    case 128: return launch_t<D, 128, M>(fp, grid, st);
+    default: return launch_t<D, 0, M>(fp, grid, st);      // any other window length: known at run time only
   }
 }
 
@@ -1170,7 +1183,7 @@ kvc_status launch_w(int W, const FastParams& fp, int grid, cudaStream_t st) {
 
 bool score_sm100_supported(const Problem& P) {
   if (P.dtype != KVC_BF16 || !P.contiguous_groups) return false;
-  if (P.w != 8 && P.w != 16 && P.w != 32 && P.w != 64 && P.w != 128) return false;
+  if (P.w < 1 || P.w > kRows) return false;
   if (P.L > kMaxFastLayers) return false;
   if (P.N >= (1LL << 30)) return false;
   FastPlan pl;

@@ -190,6 +190,27 @@ def test_tensor_core_path_shapes(Hq, Hkv, w, d, N, batch, q_pos0):
     check_all(wl, desc, cfg.budget)
 
 
+@pytest.mark.parametrize("Hq,Hkv,w,agg_task,agg_group,q_pos0", [
+    (8, 2, 24, 0, 0, None),      # five query heads of 24 rows would fit, four are there: 96 rows
+    (8, 2, 100, 0, 0, None),     # one query head of 100 rows per row tile, four row tiles
+    (4, 2, 5, 1, 1, None),       # a very short window, task mean, group max
+    (4, 2, 1, 0, 0, None),       # a single window row
+    (6, 2, 48, 1, 0, 700),       # two heads of 48 rows per tile and a short second tile; mask inside the context
+])
+def test_window_lengths_other_than_powers_of_two(Hq, Hkv, w, agg_task, agg_group, q_pos0):
+    """Any window length up to 128 runs on the tensor-core path, through the variant that reads the
+    length at run time."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("oddw", 2, Hq, Hkv, 128, 1500, w, dtype="bf16", retention=0.3, elem_std=1.0,
+                           hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    kw = dict(agg_task=agg_task, agg_group=agg_group)
+    if q_pos0 is not None:
+        kw["q_pos0"] = q_pos0
+    desc = kvc.desc_from_config(cfg, **kw)
+    check_all(wl, desc, cfg.budget)
+
+
 @pytest.mark.parametrize("scale", [2.0, 0.5])
 def test_logits_far_above_the_first_tokens(scale):
     """A large logit scale: for most window rows some token lies tens of nats above token 0, whose
