@@ -75,6 +75,7 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
                    int L, int Bt, long long N, long long budget) {
   __shared__ unsigned int sh[kRadix];
   __shared__ unsigned long long scratch[16];
+  grid_dependency_wait();
   const int b = blockIdx.y;
   unsigned int* hist_b = hist + (size_t)b * 4 * kRadix;
   for (int i = threadIdx.x; i < kRadix; i += kHistThreads) sh[i] = 0;
@@ -146,6 +147,7 @@ select_finish_kernel(const float* __restrict__ composite,
   __shared__ long long s_gt[KVC_MAX_LAYERS];
   __shared__ long long s_ge[KVC_MAX_LAYERS];
   __shared__ unsigned long long scratch[16];
+  grid_dependency_wait();
   const int b = blockIdx.x;
   const SelectState st = derive_state(hist + (size_t)b * 4 * kRadix, 4, (unsigned long long)budget, scratch);
   const uint32_t T = st.prefix;
@@ -197,12 +199,13 @@ kvc_status launch_allocate(const Problem& P, const float* composite, long long b
   if (blocks < 1) blocks = 1;
   if (budget > 0) {
     for (int pass = 0; pass < 4; ++pass) {
-      select_hist_kernel<<<dim3((unsigned)blocks, P.Bt), kHistThreads, 0, st>>>(
-          composite, hist, pass, P.L, P.Bt, P.N, budget);
+      KVC_CUDA(launch_dependent(select_hist_kernel, dim3((unsigned)blocks, P.Bt), dim3(kHistThreads), 0, st,
+                                composite, hist, pass, P.L, P.Bt, P.N, budget));
       KVC_LAUNCH_CHECK("select_hist_kernel");
     }
   }
-  select_finish_kernel<<<P.Bt, 1024, 0, st>>>(composite, hist, P.L, P.Bt, P.N, budget, n_keep, offsets);
+  KVC_CUDA(launch_dependent(select_finish_kernel, dim3(P.Bt), dim3(1024), 0, st,
+                            composite, hist, P.L, P.Bt, P.N, budget, n_keep, offsets));
   KVC_LAUNCH_CHECK("select_finish_kernel");
   return KVC_OK;
 }

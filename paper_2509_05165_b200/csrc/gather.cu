@@ -40,6 +40,7 @@ gather_kernel(GatherParams P, LayerPtrs kp, LayerPtrs vp, const int32_t* __restr
               const int32_t* __restrict__ n_keep, const long long* __restrict__ offsets,
               uint4* __restrict__ k_out, uint4* __restrict__ v_out) {
   __shared__ long long s_off[KVC_MAX_LAYERS + 1];
+  grid_dependency_wait();
   const int b = blockIdx.y;
   for (int i = threadIdx.x; i <= P.L; i += kGatherThreads) s_off[i] = offsets[(long long)b * (P.L + 1) + i];
   __syncthreads();
@@ -105,8 +106,9 @@ kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& 
   const long long cap = 148LL * 128;   // measured best among 8 to 256 CTAs per SM's worth of grid
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  gather_kernel<<<dim3((unsigned)blocks, P.Bt), kGatherThreads, 0, st>>>(
-      gp, k, v, idx, n_keep, offsets, reinterpret_cast<uint4*>(k_out), reinterpret_cast<uint4*>(v_out));
+  KVC_CUDA(launch_dependent(gather_kernel, dim3((unsigned)blocks, P.Bt), dim3(kGatherThreads), 0, st,
+                            gp, k, v, idx, n_keep, offsets, reinterpret_cast<uint4*>(k_out),
+                            reinterpret_cast<uint4*>(v_out)));
   KVC_LAUNCH_CHECK("gather_kernel");
   return KVC_OK;
 }

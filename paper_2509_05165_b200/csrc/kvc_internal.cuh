@@ -53,6 +53,32 @@ void count_launch(int n = 1);
     if (_s != KVC_OK) return _s;                              \
   } while (0)
 
+// Programmatic dependent launch: the kernel may be scheduled while the kernel before it in the
+// stream is still draining, which hides its launch latency.  Every kernel launched this way
+// calls grid_dependency_wait() before it touches global memory: the call returns once the
+// preceding kernel has completed and its writes are visible (and so, transitively, all earlier
+// work in the stream).
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // Host-side validation shared by the entry points that live outside kvc_api.cu.
 kvc_status resolve_desc(const kvc_desc* d, Problem* P);
 kvc_status require_budget(const Problem& P, long long budget);

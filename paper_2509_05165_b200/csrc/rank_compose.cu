@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(kSortThreads, 4)
 sort_count_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
                   uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
   __shared__ uint32_t hist[kRadix];
+  grid_dependency_wait();
   const long long seg = blockIdx.x / tiles;
   const int tile = (int)(blockIdx.x - seg * tiles);
   const PassIo io = pass_io(buf, idx_out, pass, seg * N);
@@ -118,6 +119,7 @@ sort_scatter_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* 
   __shared__ uint32_t stage_k[kTileItems];        // the tile, reordered by digit, before it goes out
   __shared__ int32_t stage_v[kTileItems];
 
+  grid_dependency_wait();
   const long long seg = blockIdx.x / tiles;
   const int tile = (int)(blockIdx.x - seg * tiles);
   const PassIo io = pass_io(buf, idx_out, pass, seg * N);
@@ -224,6 +226,7 @@ sort_scatter_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* 
 // Mean: heads added in ascending order in fp32, one division at the end.
 __global__ void compose_kernel(const uint32_t* __restrict__ keys, float* __restrict__ composite,
                                int Hkv, long long N, long long total, int agg_head) {
+  grid_dependency_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const long long lb = i / N, kk = i - lb * N;
@@ -270,14 +273,16 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
     return KVC_ERR_UNSUPPORTED;
   }
   for (int pass = 0; pass < 4; ++pass) {
-    sort_count_kernel<<<(unsigned)blocks, kSortThreads, 0, st>>>(scores, buf, idx, counts, P.N, tiles, pass);
+    KVC_CUDA(launch_dependent(sort_count_kernel, dim3((unsigned)blocks), dim3(kSortThreads), 0, st,
+                              scores, buf, idx, counts, P.N, tiles, pass));
     KVC_LAUNCH_CHECK("sort_count_kernel");
-    sort_scatter_kernel<<<(unsigned)blocks, kSortThreads, 0, st>>>(scores, buf, idx, counts, P.N, tiles, pass);
+    KVC_CUDA(launch_dependent(sort_scatter_kernel, dim3((unsigned)blocks), dim3(kSortThreads), 0, st,
+                              scores, buf, idx, counts, P.N, tiles, pass));
     KVC_LAUNCH_CHECK("sort_scatter_kernel");
   }
   const long long total = (long long)P.L * P.Bt * P.N;
-  compose_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(buf.keys_b, composite, P.Hkv, P.N,
-                                                                 total, P.agg_head);
+  KVC_CUDA(launch_dependent(compose_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
+                            buf.keys_b, composite, P.Hkv, P.N, total, P.agg_head));
   KVC_LAUNCH_CHECK("compose_kernel");
   return KVC_OK;
 }

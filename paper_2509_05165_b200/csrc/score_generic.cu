@@ -243,6 +243,7 @@ score_emit_kernel(ScoreParams P, GroupMap gm, LayerPtrs qp, LayerPtrs kp,
 // Eq. 15 from the tiles' partial aggregates (sum or max over the tile's query heads), in tile order.
 __global__ void score_augment_kernel(float* __restrict__ s, const float* __restrict__ parts, int row_tiles,
                                      int G, int agg_group, int augment, int Hkv, long long N, long long total) {
+  grid_dependency_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const long long lb = i / N, c = i - lb * N;
@@ -309,8 +310,8 @@ kvc_status launch_score_augment(const Problem& P, float* scores, const float* pa
                                 cudaStream_t st) {
   if (!P.augment && row_tiles <= 1) return KVC_OK;
   const long long total = (long long)P.L * P.Bt * P.N;
-  score_augment_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
-      scores, parts, row_tiles, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total);
+  KVC_CUDA(launch_dependent(score_augment_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
+                            scores, parts, row_tiles, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total));
   KVC_LAUNCH_CHECK("score_augment_kernel");
   return KVC_OK;
 }

@@ -547,6 +547,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dependency_wait();      // everything above overlapped the end of the kernel before this one
 
   // this CTA's share of the runs and the length of its sequence
   // (the host keeps all of these below 2^31)
@@ -1162,7 +1163,7 @@ kvc_status launch_t(const FastParams& fp, int grid, cudaStream_t st) {
     KVC_CUDA(cudaFuncSetAttribute(score_sm100_kernel<D, W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal));
     attr_set = true;
   }
-  score_sm100_kernel<D, W, M><<<grid, kFastThreads, SL::kTotal, st>>>(fp);
+  KVC_CUDA(launch_dependent(score_sm100_kernel<D, W, M>, dim3(grid), dim3(kFastThreads), (size_t)SL::kTotal, st, fp));
   KVC_LAUNCH_CHECK("score_sm100_kernel");
   return KVC_OK;
 }
