@@ -1040,14 +1040,24 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 // 2^(logit - ref) is then at least about 1, so fixed point with 20 fractional bits keeps it.
 // ------------------------------------------------------------------------------------------------
 struct RefParams {
-  int Bt, Hkv, G, HPT, QT, w, d;
+  int Bt, Hkv, G, HPT, QT, w, d, NG;
+  unsigned long long* acc;     // [U][128]: cleared here
+  int* group_counter;          // [U][NG], int* unit_counter [U], unsigned* lse2 [U][128]: preset here
+  int* unit_counter;
+  unsigned int* lse2;
   long long qs0, qs1, qs2, kvs0, kvs1;
   float sl2e;
 };
 
 __global__ void __launch_bounds__(kRows)
 score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ ref) {
+  grid_dependency_wait();
   const int u = blockIdx.x, row = threadIdx.x;
+  // the unit's exchange state: empty words, counters at -1, log-sum-exp slots "not there yet"
+  P.acc[(long long)u * kRows + row] = 0ull;
+  P.lse2[(long long)u * kRows + row] = 0xffffffffu;
+  if (row < P.NG) P.group_counter[(long long)u * P.NG + row] = -1;
+  if (row == 0) P.unit_counter[u] = -1;
   const int uh = u / P.QT, qt = u - uh * P.QT;
   const int lb = uh / P.Hkv, h = uh - lb * P.Hkv;
   const int l = lb / P.Bt, b = lb - l * P.Bt;
@@ -1223,8 +1233,6 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
     if (!encode_map(&fp.q_maps[l], q.p[l], qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
   }
   char* w = reinterpret_cast<char*>(ws);
-  // counters start at -1 and the log-sum-exp slots at the "not there yet" pattern: all bits set
-  KVC_CUDA(cudaMemsetAsync(w + pl.off_sync, 0xff, pl.sync_bytes, st));
 
   fp.partial = reinterpret_cast<float4*>(w + pl.off_partial);
   fp.group_partial = reinterpret_cast<float4*>(w + pl.off_group);
@@ -1235,12 +1243,13 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   float* ref = reinterpret_cast<float*>(w + pl.off_ref);
   fp.ref = ref;
   {
-    KVC_CUDA(cudaMemsetAsync(fp.acc, 0, (size_t)pl.U * kRows * sizeof(unsigned long long), st));
     RefParams rp;
+    rp.NG = pl.NG; rp.acc = fp.acc; rp.group_counter = fp.group_counter; rp.unit_counter = fp.unit_counter;
+    rp.lse2 = fp.lse2;
     rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.w = P.w; rp.d = P.d;
     rp.qs0 = P.qs[0]; rp.qs1 = P.qs[1]; rp.qs2 = P.qs[2]; rp.kvs0 = P.kvs[0]; rp.kvs1 = P.kvs[1];
     rp.sl2e = P.scale * kLog2eF;
-    score_ref_kernel<<<pl.U, kRows, 0, st>>>(rp, q, k, ref);
+    KVC_CUDA(launch_dependent(score_ref_kernel, dim3(pl.U), dim3(kRows), 0, st, rp, q, k, ref));
     KVC_LAUNCH_CHECK("score_ref_kernel");
   }
   fp.status = device_status;
