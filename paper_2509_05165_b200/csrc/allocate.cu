@@ -70,6 +70,14 @@ __device__ inline SelectState derive_state(const unsigned int* __restrict__ hist
   return s;
 }
 
+// Clears the histograms of all passes (a kernel rather than a memset, so that it can be launched
+// as a programmatic dependent of whatever ran before).
+__global__ void __launch_bounds__(1024)
+select_clear_kernel(unsigned int* __restrict__ hist) {
+  grid_dependency_wait();
+  hist[(size_t)blockIdx.x * 4 * kRadix + threadIdx.x] = 0u;
+}
+
 __global__ void __launch_bounds__(kHistThreads)
 select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict__ hist, int pass,
                    int L, int Bt, long long N, long long budget) {
@@ -191,7 +199,8 @@ kvc_status launch_allocate(const Problem& P, const float* composite, long long b
     return KVC_ERR_WORKSPACE;
   }
   unsigned int* hist = reinterpret_cast<unsigned int*>(ws);
-  KVC_CUDA(cudaMemsetAsync(hist, 0, (size_t)P.Bt * 4 * kRadix * sizeof(unsigned int), st));
+  KVC_CUDA(launch_dependent(select_clear_kernel, dim3(P.Bt), dim3(4 * kRadix), 0, st, hist));
+  KVC_LAUNCH_CHECK("select_clear_kernel");
   const long long total = (long long)P.L * P.N;
   const long long tile = (long long)kHistThreads * kItemsPerThread;
   long long blocks = (total + tile - 1) / tile;
