@@ -250,7 +250,7 @@ def aggregate_tokens_per_s(cfg, world, ms_per_step):
 # summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of a 4-layer capture,
 # scaled by 8 to the 32 layers of the workload: the traffic is proportional to the layers).
 # None for any other workload, and to be reset to None whenever the kernel changes.
-SCORE_TRAFFIC_BYTES = {"llama8b_32k": 8 * (273694720 + 7339008)}   # 2.25 GB: K leaves HBM once (1.04x algorithmic)
+SCORE_TRAFFIC_BYTES = {"llama8b_32k": 8 * (273443072 + 8006912)}   # 2.25 GB: K leaves HBM once (1.04x algorithmic)
 
 
 def workload_config(cfg, world):
