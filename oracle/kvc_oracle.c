@@ -127,6 +127,9 @@ int oracle_score_layer(const float* q, const float* k, int32_t Hq, int32_t Hkv,
     int32_t h = q_to_kv ? q_to_kv[j] : j / G;
     double* A = (double*)malloc(sizeof(double) * (size_t)w * (size_t)N);
     if (!A) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
       failed = 1;
       continue;
     }
@@ -386,8 +389,12 @@ int oracle_compress(const float* q, const float* k, const uint8_t* k_raw,
     for (int32_t h = 0; h < Hkv; ++h) {
       if (oracle_rank(S + l * per_layer + (int64_t)h * N, N,
                       idx + l * (int64_t)per_layer + (int64_t)h * N,
-                      S_sorted + (int64_t)h * N))
+                      S_sorted + (int64_t)h * N)) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
         bad = 1;
+      }
     }
     if (bad) rc = -1;
     if (rc == 0) oracle_compose(S_sorted, Hkv, N, agg_head, I + (int64_t)l * N);

@@ -18,3 +18,17 @@ def oracle():
 
     _oracle.build()
     return _oracle
+
+
+def pytest_terminal_summary(terminalreporter):
+    """The parity reports of the GPU tests (score error, order differences with their oracle gaps,
+    tie margins, allocation differences), printed whether or not output is captured."""
+    try:
+        import parity
+    except Exception:  # noqa: BLE001
+        return
+    if not parity.REPORTS:
+        return
+    terminalreporter.section("parity reports (GPU vs the all-double oracle)")
+    for name, fields in parity.REPORTS:
+        terminalreporter.write_line("%s: %s" % (name, ", ".join("%s=%s" % kv for kv in fields.items())))
