@@ -113,9 +113,17 @@ KVC_API kvc_status kvc_workspace_size(const kvc_desc* desc, int64_t budget, size
  * q, k: HOST arrays of n_layers device pointers.  scores: [L, batch, Hkv, N] fp32, dense.
  * bf16 inputs are multiplied exactly and accumulated in fp32; the attention tensor A is
  * never written to memory.
+ *
+ * Conditions that only the device can detect (KVC_ERR_TIMEOUT, see kvc_compress) are reported in
+ * an int32 inside the workspace, at the byte offset kvc_score_status_offset() returns: 0 after a
+ * good run.  Read it once the stream has finished the call; the scores are meaningless otherwise.
  */
 KVC_API kvc_status kvc_score(const kvc_desc* desc, const void* const* q, const void* const* k,
                      float* scores, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Byte offset, inside the workspace handed to kvc_score, of the int32 device status word that call
+ * writes (host call; depends on the problem only). */
+KVC_API kvc_status kvc_score_status_offset(const kvc_desc* desc, size_t* offset);
 
 /*
  * Ranking and composite tokens (Sec. 3.3).  For every (l, b, h):
@@ -182,6 +190,14 @@ KVC_API kvc_status kvc_gather(const kvc_desc* desc, const void* const* k, const 
  * The whole pass, stream-ordered.  idx_out [L, batch, Hkv, N], scores_out [L, batch, Hkv, N] and
  * composite_out [L, batch, N] may be NULL (the workspace then holds them).  device_status, if
  * not NULL, receives KVC_OK or a negative kvc_status detected on the device.
+ *
+ * The bf16 scoring kernel (kvc_score and kvc_compress) is one persistent grid of a CTA per SM
+ * whose CTAs exchange the softmax statistics through global memory, so all of them have to be
+ * resident at the same time.  Give it the GPU to itself: while other work holds SMs (another
+ * stream's kernels, a second kvc_score / kvc_compress in flight, an MPS share smaller than the
+ * device) its CTAs may wait for CTAs that cannot start.  Such a wait is bounded (2 s): the kernel
+ * then stops, the status word is KVC_ERR_TIMEOUT, the outputs of the call are meaningless, and
+ * the context stays usable.  Calls on one stream, or ordered by events, never overlap.
  */
 KVC_API kvc_status kvc_compress(const kvc_desc* desc, const void* const* q, const void* const* k,
                         const void* const* v, int64_t budget, void* k_out, void* v_out,
@@ -195,6 +211,13 @@ KVC_API const char* kvc_last_error(void);
 /* Number of kernels the library has launched on this thread since the last call with reset != 0
  * (a host-side counter for benchmarks; it does not touch the device). */
 KVC_API int64_t kvc_launch_count(int32_t reset);
+
+/* Test hook, not for production use: sets the bound of the scoring kernel's device-side waits
+ * (nanoseconds; <= 0 restores the default of 2 s) and names one work unit of that kernel -- (layer,
+ * sequence, KV head, row tile) numbered in that order -- whose softmax statistics are withheld, so
+ * that the waits for them run into the bound and the call ends with KVC_ERR_TIMEOUT in its status
+ * word (-1: none).  Process-wide; takes effect at the next launch. */
+KVC_API void kvc_debug_score_hooks(int64_t wait_limit_ns, int32_t withhold_unit);
 
 /* Library version as major * 10000 + minor * 100 + patch. */
 KVC_API int32_t kvc_version(void);

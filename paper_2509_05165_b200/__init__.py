@@ -20,7 +20,9 @@ from .binding import (  # noqa: F401
     kvc_gather,
     kvc_last_error,
     kvc_launch_count,
+    kvc_debug_score_hooks,
     kvc_score,
+    kvc_score_status_offset,
     kvc_version,
     kvc_workspace_size,
     library_path,

@@ -66,6 +66,10 @@ def _load():
     lib.kvc_workspace_size.restype = C.c_int
     lib.kvc_score.argtypes = [dp, vp, vp, vp, vp, sz, vp]
     lib.kvc_score.restype = C.c_int
+    lib.kvc_score_status_offset.argtypes = [dp, C.POINTER(sz)]
+    lib.kvc_score_status_offset.restype = C.c_int
+    lib.kvc_debug_score_hooks.argtypes = [i64, i32]
+    lib.kvc_debug_score_hooks.restype = None
     lib.kvc_compose.argtypes = [dp, vp, vp, vp, vp, sz, vp]
     lib.kvc_compose.restype = C.c_int
     lib.kvc_allocate.argtypes = [dp, vp, i64, vp, vp, vp, sz, vp]
@@ -135,6 +139,19 @@ def kvc_score(desc, q: Sequence[torch.Tensor], k: Sequence[torch.Tensor], scores
     wp, wb = _ws(workspace)
     _check(_load().kvc_score(C.byref(desc), _ptr_array(q), _ptr_array(k), _dptr(scores), wp, wb,
                              _stream(stream)))
+
+
+def kvc_score_status_offset(desc: KvcDesc) -> int:
+    """Byte offset, in the workspace given to ``kvc_score``, of that call's int32 device status."""
+    out = C.c_size_t(0)
+    _check(_load().kvc_score_status_offset(C.byref(desc), C.byref(out)))
+    return int(out.value)
+
+
+def kvc_debug_score_hooks(wait_limit_ns: int = 0, withhold_unit: int = -1) -> None:
+    """Test hook: bound of the scoring kernel's device-side waits, and a unit whose statistics
+    are withheld so that those waits expire.  The defaults restore normal operation."""
+    _load().kvc_debug_score_hooks(int(wait_limit_ns), int(withhold_unit))
 
 
 def kvc_compose(desc, scores, idx, composite, workspace, stream=None) -> None:

@@ -26,14 +26,17 @@ kvc_status check_cuda(cudaError_t e, const char* what) {
 
 void count_launch(int n) { g_launches += n; }
 
-size_t score_workspace_bytes(const Problem& P) {
+// Scratch of the scoring kernels; kvc_score keeps its device status word right behind it.
+static size_t score_scratch_bytes(const Problem& P) {
   size_t a = score_generic_workspace_bytes(P);
   if (score_sm100_supported(P)) {
     const size_t b = score_sm100_workspace_bytes(P);
     if (b > a) a = b;
   }
-  return a;
+  return align_up(a);
 }
+
+size_t score_workspace_bytes(const Problem& P) { return score_scratch_bytes(P) + 256; }
 
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
                         float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -253,7 +256,19 @@ kvc_status kvc_score(const kvc_desc* d, const void* const* q, const void* const*
   KVC_REQUIRE(scores != nullptr, KVC_ERR_INVALID_ARG, "scores is NULL");
   if ((s = check_ws(ws, ws_bytes, score_workspace_bytes(P))) != KVC_OK) return s;
   if ((s = check_device()) != KVC_OK) return s;
-  return launch_score(P, gm, qp, kp, scores, nullptr, ws, ws_bytes, (cudaStream_t)stream);
+  // conditions detected on the device are reported in a word behind the scratch (kvc_score_status_offset)
+  int* status = reinterpret_cast<int*>(reinterpret_cast<char*>(ws) + score_scratch_bytes(P));
+  KVC_CUDA(cudaMemsetAsync(status, 0, sizeof(int), (cudaStream_t)stream));
+  return launch_score(P, gm, qp, kp, scores, status, ws, score_scratch_bytes(P), (cudaStream_t)stream);
+}
+
+kvc_status kvc_score_status_offset(const kvc_desc* d, size_t* offset) {
+  Problem P; GroupMap gm;
+  const kvc_status s = resolve(d, &P, &gm);
+  if (s != KVC_OK) return s;
+  KVC_REQUIRE(offset != nullptr, KVC_ERR_INVALID_ARG, "offset is NULL");
+  *offset = score_scratch_bytes(P);
+  return KVC_OK;
 }
 
 kvc_status kvc_compose(const kvc_desc* d, const float* scores, int32_t* idx, float* composite,

@@ -9,20 +9,20 @@
 //   exchange             a run of RT consecutive tiles of one (layer, sequence, KV head) unit
 //                        yields one (reference, sum) per row.  The short way: every row has a
 //                        fixed reference (its logit against token 0, from a small kernel that
-//                        runs first) and one 64-bit word; the pass-1 epilogue rescales the run's
-//                        sum to that reference, converts it to fixed point (2^-20) and adds it,
-//                        together with an arrival count in the top byte, with one integer
-//                        reduction.  Integer addition makes the total independent of the order
-//                        of arrival, and sum and count travel in one word, so a reader needs no
-//                        fence: the word is complete when its count equals the unit's runs.
-//                        That is two round trips to L2 between the last pass-1 tile of a unit
-//                        and its first pass-2 tile.  The long way, always taken as well: the
-//                        run's record of (reference, sum) per row goes to global memory and is
-//                        counted into its group of kGroupRuns runs; every group and every unit
-//                        has a fixed folding CTA (round-robin) whose exchange warp waits for the
-//                        count and folds in a fixed order, down to the rows' log-sum-exp.  Pass 2
-//                        uses it for the rows whose word says that some run's sum did not fit
-//                        the fixed-point range (a token about 14 nats above token 0).
+//                        runs first) and one 64-bit word; the run's sum is rescaled to that
+//                        reference, converted to fixed point (2^-20) and added, together with an
+//                        arrival count in the top byte, with one integer reduction.  Integer
+//                        addition makes the total independent of the order of arrival, and sum
+//                        and count travel in one word, so a reader needs no fence: the word is
+//                        complete when its count equals the unit's runs.  That is two round
+//                        trips to L2 between the last pass-1 tile of a unit and its first pass-2
+//                        tile.  The long way, always taken as well: the run's record of
+//                        (reference, sum) per row goes to global memory and is counted into its
+//                        group of kGroupRuns runs; every group and every unit has a fixed folding
+//                        CTA (round-robin) whose exchange warp waits for the count and folds in
+//                        a fixed order, down to the rows' log-sum-exp.  Pass 2 uses it for the
+//                        rows whose word says that some run's sum did not fit the fixed-point
+//                        range (a token about 14 nats above token 0).
 //   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
 //                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
 //                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
@@ -33,23 +33,28 @@
 // A unit is a (layer, sequence, KV head, row tile): the G x w window rows of a KV head are cut
 // into row tiles of at most 128 rows (whole query heads), so that any GQA group / window size
 // with w <= 128 runs here (w = 8, 16, 32, 64, 128 as compile-time specialisations, any other
-// length through one variant that reads it at run time); with more than one row tile the pass-2 results are partial group
-// aggregates that the Eq. 16 kernel combines in a fixed order.
+// length through one variant that reads it at run time); with more than one row tile the
+// pass-2 results are partial group aggregates that the Eq. 16 kernel combines in a fixed order.
 //
 // Every CTA walks one static sequence that alternates a pass-1 tile with a pass-2 tile; the
 // pass-2 stream trails the pass-1 stream by `shift` tiles (two runs where a unit has no more
-// runs than there are CTAs: 38 MB of K at 148 CTAs, which L2 still holds).  A pass-2 tile only ever waits for
-// pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot deadlock while all
-// CTAs are resident.  Every wait (mbarrier or global flag) is bounded; on expiry the kernel
-// records KVC_ERR_TIMEOUT, stops computing and drains.
+// runs than there are CTAs: 38 MB of K at 148 CTAs, which L2 still holds).  A pass-2 tile only
+// ever waits for pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot
+// deadlock while all CTAs are resident (the host checks that they can be).  Every wait
+// (mbarrier, shared-memory counter or global flag) is bounded; on expiry the kernel records
+// KVC_ERR_TIMEOUT, stops computing and drains.
 //
 // Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch); warp 1 = MMA
-// issuer of pass 1 and TMEM owner; warp 2 = MMA issuer of pass 2 (two issuers, because the
-// waits, commits and bookkeeping around a tile cost one thread more time than the tile's MMAs
-// take, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-7 =
-// pass-2 epilogue; warps 8-15 = pass-1 epilogue (two warpgroups, each takes one half of every
-// tile's columns).
+// issuer of pass 1 and TMEM owner; warp 2 = MMA issuer of pass 2 (two issuers: issuing the eight
+// MMAs of a tile takes a thread about 420 clocks, a commit about 50 and every barrier wait
+// about 100 even when it succeeds at once, which together is more than the 512 tensor clocks of
+// the tile, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-7 =
+// pass-2 epilogue; warps 8-15 = pass-1 epilogue (two groups of four warps, each takes one half
+// of every tile's columns).
 #include <cuda.h>
+
+#include <atomic>
+#include <mutex>
 
 #include "kvc_internal.cuh"
 
@@ -64,21 +69,6 @@
 #endif
 
 namespace kvc {
-#ifdef KVC_SCORE_TRACE
-// Optional trace (debug builds only): per CTA, SM clocks each role spent in each kind of wait.
-__device__ unsigned long long g_score_trace[160 * 24];
-#define KVC_TR_DECL(...) long long __VA_ARGS__
-#define KVC_TR(acc, stmt) do { const long long _t0 = clock64(); stmt; acc += clock64() - _t0; } while (0)
-#define KVC_TR_SINCE(acc, start) acc += clock64() - (start)
-#define KVC_TR_PUT(i, v) g_score_trace[blockIdx.x * 24 + (i)] = (unsigned long long)(v)
-#define KVC_TR_NOW() clock64()
-#else
-#define KVC_TR_SINCE(acc, start)
-#define KVC_TR_DECL(...)
-#define KVC_TR(acc, stmt) do { stmt; } while (0)
-#define KVC_TR_PUT(i, v)
-#define KVC_TR_NOW() 0ll
-#endif
 namespace {
 
 constexpr int kTile = 128;            // tokens per tile = MMA M = MMA N
@@ -90,7 +80,7 @@ constexpr int kQSlots = 3;
 constexpr int kPrefetch = KVC_SCORE_PREFETCH;
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kRescaleLimit = 1.8446744e19f;               // 2^64: a chunk sum beyond it restarts with a new reference
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
 
 constexpr int kMaxFastLayers = 112;   // 2 tensor maps per layer must fit the 32 KB kernel-parameter space
 
@@ -118,6 +108,9 @@ struct FastParams {
   int shift;                   // tiles by which the pass-2 stream trails the pass-1 stream
   float sl2e;                  // scale * log2(e)
   int agg_group;
+  unsigned long long wait_limit_ns;   // bound of every device-side wait
+  int withhold_unit;           // test hook: the statistics of this unit are never sent (-1: none), so that
+                               // the waits for them run into their bound
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -149,23 +142,45 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the abort word is set or the time limit expires (and sets it).
-// The retry loop is kept out of line: the kernel's hot loops have to stay small enough for the
-// instruction cache, which sixteen warps in six different roles share.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+// Per-CTA control block in shared memory.
+struct Ctl {
+  int abort;                       // set by the first wait of this CTA that gives up
+  int pad;
+  unsigned long long limit_ns;     // bound of every wait
+  const int* grid_status;          // the device status word (may be null): non-zero once any CTA gave up
+};
+// Called from the slow part of every wait loop: has this CTA, or any other, given up, or has this
+// wait lasted longer than the bound?  (Then it marks the CTA as aborted.)
+__device__ __noinline__ bool give_up(volatile Ctl* ctl, unsigned long long t0) {
+  if (ctl->abort) return true;
+  const int* gs = ctl->grid_status;
+  if (gs != nullptr && *reinterpret_cast<const volatile int*>(gs) != 0) { ctl->abort = 1; return true; }
+  if (globaltimer_ns() - t0 > ctl->limit_ns) { ctl->abort = 1; return true; }
+  return false;
+}
+// Bounded wait.  Returns false when the CTA has given up (see give_up).  The retry loop is kept
+// out of line: the kernel's hot loops have to stay small enough for the instruction cache.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile Ctl* ctl) {
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
   while (!mbar_try(bar, parity)) {
-    if ((++spins & 1023u) == 0) {
-      if (*abort_word) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; return false; }
-    }
+    if ((++spins & 1023u) == 0 && give_up(ctl, t0)) return false;
   }
   return true;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile Ctl* ctl) {
   if (mbar_try(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_word);
+  return mbar_wait_slow(bar, parity, ctl);
+}
+// The same for a copy or an MMA that has been issued and therefore completes whatever the rest
+// of the grid does: only the time bound ends this wait early, not the abort flag.
+__device__ __noinline__ bool mbar_wait_issued(uint32_t bar, uint32_t parity, volatile Ctl* ctl) {
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 1023u) == 0 && globaltimer_ns() - t0 > ctl->limit_ns) { ctl->abort = 1; return false; }
+  }
+  return true;
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3, unsigned long long policy) {
@@ -376,14 +391,15 @@ struct SmemLayout {
   static constexpr int kBarTEmpty = kBarTFull + 32;
   static constexpr int kBarQFull = kBarTEmpty + 32;            // kQSlots x 8
   static constexpr int kBarQFree = kBarQFull + 8 * kQSlots;
-  static constexpr int kTmemSlot = kBarQFree + 8 * kQSlots;    // 4 B (+ padding)
-  static constexpr int kAbort = kTmemSlot + 8;                 // 4 B
-  static constexpr int kFlushed = kAbort + 8;                  // 4 B: warps that have written a run's record
+  static constexpr int kBarMmaDone = kBarQFree + 8 * kQSlots;  // 2 x 8
+  static constexpr int kTmemSlot = kBarMmaDone + 16;           // 4 B (+ padding)
+  static constexpr int kCtl = kTmemSlot + 8;                   // Ctl, 24 B
+  static constexpr int kFlushed = kCtl + 24;                   // 4 B: warps that have written a run's record
   static constexpr int kNegLse = (kFlushed + 8 + 15) / 16 * 16;  // 128 floats, read as 16-byte vectors:
                                                                // -log-sum-exp of the pass-2 unit
   static constexpr int kStats = kNegLse + kRows * 4;           // 128 rows x float2: the upper half's statistics
   static constexpr int kTotal = kStats + kRows * 8;
-  static_assert(kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
+  static_assert(kCtl % 8 == 0 && kNegLse % 16 == 0 && kStats % 8 == 0 && kTotal <= 232448, "shared-memory layout");
 };
 
 // The pushed statistics of one row (see FastParams::acc).
@@ -394,30 +410,24 @@ constexpr unsigned long long kAccSumMask = kAccOverflow - 1;
 
 // Bounded poll of a row's pushed statistics until all `runs` runs of the unit have arrived.
 __device__ __noinline__ unsigned long long poll_acc_slow(const unsigned long long* src, unsigned int runs,
-                                                         volatile int* abort_word) {
+                                                         volatile Ctl* ctl) {
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
   unsigned long long v;
   while ((unsigned int)((v = ld_relaxed_u64(src)) >> 56) != runs) {
     __nanosleep(100);
-    if ((++spins & 255u) == 0) {
-      if (*abort_word) break;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
-    }
+    if ((++spins & 255u) == 0 && give_up(ctl, t0)) break;
   }
   return v;
 }
 
 // Bounded poll of a log-sum-exp slot (the value itself is the flag).
-__device__ __noinline__ uint32_t poll_lse_slow(const unsigned int* src, volatile int* abort_word) {
+__device__ __noinline__ uint32_t poll_lse_slow(const unsigned int* src, volatile Ctl* ctl) {
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0, bits;
   while ((bits = ld_relaxed_u32(src)) == 0xffffffffu) {
     __nanosleep(100);
-    if ((++spins & 255u) == 0) {
-      if (*abort_word) break;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; break; }
-    }
+    if ((++spins & 255u) == 0 && give_up(ctl, t0)) break;
   }
   return bits;
 }
@@ -515,13 +525,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sbase = smem_u32(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  volatile int* abort_word = reinterpret_cast<volatile int*>(smem + SL::kAbort);
+  volatile Ctl* ctl = reinterpret_cast<volatile Ctl*>(smem + SL::kCtl);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SL::kTmemSlot);
-
-  if ((sbase & 1023u) != 0) {          // the swizzled tiles need a 1024-byte aligned base
-    if (threadIdx.x == 0 && P.status) atomicCAS(P.status, 0, (int)KVC_ERR_CUDA);
-    return;
-  }
 
   auto bar_kfull = [&](int s) { return sbase + SL::kBarKFull + 8 * s; };
   auto bar_kempty = [&](int s) { return sbase + SL::kBarKEmpty + 8 * s; };
@@ -529,12 +534,18 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   auto bar_tempty = [&](int b) { return sbase + SL::kBarTEmpty + 8 * b; };
   auto bar_qfull = [&](int q) { return sbase + SL::kBarQFull + 8 * q; };
   auto bar_qfree = [&](int q) { return sbase + SL::kBarQFree + 8 * q; };
+  auto bar_mma_done = [&](int p) { return sbase + SL::kBarMmaDone + 8 * p; };
 
+  const bool aligned = (sbase & 1023u) == 0;     // the swizzled tiles need a 1024-byte aligned base
   if (threadIdx.x == 0) {
     for (int s = 0; s < SL::kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 2); }
+    // the accumulators of pass 1 are read by eight warps (two column halves), those of pass 2 by four
     for (int b = 0; b < 4; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), b < 2 ? 8 : 4); }
     for (int q = 0; q < kQSlots; ++q) { mbar_init(bar_qfull(q), 1); mbar_init(bar_qfree(q), 2); }
-    *abort_word = 0;
+    mbar_init(bar_mma_done(0), 1); mbar_init(bar_mma_done(1), 1);
+    ctl->abort = 0;
+    ctl->limit_ns = P.wait_limit_ns;
+    ctl->grid_status = P.status;
     *reinterpret_cast<volatile int*>(smem + SL::kFlushed) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -551,7 +562,11 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 
   // this CTA's share of the runs and the length of its sequence
   // (the host keeps all of these below 2^31)
-  const int my_runs = (P.total_runs > blockIdx.x) ? (int)((P.total_runs - blockIdx.x + P.grid - 1) / P.grid) : 0;
+  int my_runs = (P.total_runs > blockIdx.x) ? (int)((P.total_runs - blockIdx.x + P.grid - 1) / P.grid) : 0;
+  if (!aligned) {
+    if (threadIdx.x == 0 && P.status) atomicCAS(P.status, 0, (int)KVC_ERR_CUDA);
+    my_runs = 0;               // nothing is computed; the teardown below still frees the TMEM columns
+  }
   const int my_tiles = my_runs * P.RT;                  // stream length (some positions hold no tile)
   const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
   const uint32_t q_bytes = (uint32_t)(P.HPT * P.w) * D * 2;   // the whole box arrives (rows outside the tensor as zeros)
@@ -563,7 +578,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       unsigned long long pol_stream, pol_keep;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-      KVC_TR_DECL(w_q = 0, w_k = 0, w_s = KVC_TR_NOW());
       Ring kr = {0, 0}, qr = {0, 0};   // next K stage / Q slot to fill; phase = parity of the fill count / ring size
       int nk = 0, qc = 0;              // K tiles / Q tiles issued (saturating small counts are all that is needed)
       bool ok = true;
@@ -588,7 +602,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           Cursor& c = cur[pass];
           if (c.valid(P)) {
             if (c.t == 0) {                                    // a new run: its Q goes into the next ring slot
-              KVC_TR(w_q, if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), abort_word));
+              if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), ctl);
               if (ok) {
                 mbar_expect_tx(bar_qfull(qr.i), q_bytes);
                 for (int hf = 0; hf < SL::kHalves; ++hf)
@@ -598,7 +612,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 if (qc < kQSlots) ++qc;
               }
             }
-            KVC_TR(w_k, if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), abort_word));
+            if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), ctl);
             if (ok) {
               mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
               // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
@@ -613,19 +627,19 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           if (pass == 0) prefetch_next();
         }
       }
-      KVC_TR_PUT(0, w_q); KVC_TR_PUT(1, w_k); KVC_TR_PUT(2, KVC_TR_NOW() - w_s);
-      // drain: every issued copy must have landed before the CTA's shared memory is released.
+      // drain: every issued copy must have landed before the CTA's shared memory is released
+      // (an issued copy always completes, so these waits do not take the abort shortcut).
       // The last fill of stage i is complete once its full barrier has left the phase of that fill.
       for (int n = 0; n < nk; ++n) {
         // walk the ring backwards from the slot before kr
         int i2 = kr.i - 1 - n, ph = kr.phase;
         if (i2 < 0) { i2 += SL::kStages; ph ^= 1; }
-        mbar_wait(bar_kfull(i2), (uint32_t)ph, abort_word);
+        mbar_wait_issued(bar_kfull(i2), (uint32_t)ph, ctl);
       }
       for (int n = 0; n < qc; ++n) {
         int i2 = qr.i - 1 - n, ph = qr.phase;
         if (i2 < 0) { i2 += kQSlots; ph ^= 1; }
-        mbar_wait(bar_qfull(i2), (uint32_t)ph, abort_word);
+        mbar_wait_issued(bar_qfull(i2), (uint32_t)ph, ctl);
       }
     }
   } else if (warp < 3) {
@@ -643,7 +657,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       int nt = 0;                      // tiles issued (saturating at 2)
       int cur_slot = 0;
       bool ok = true;
-      KVC_TR_DECL(m_q = 0, m_ko = 0, m_kx = 0, m_t = 0, m_i = 0, m_s = KVC_TR_NOW());
       Cursor cur[2];
       cur[0].init(P); cur[1].init(P);
       for (int i = 0; i < n_steps && ok; ++i) {
@@ -654,17 +667,15 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           Cursor& c = cur[pass];
           if (c.valid(P)) {
             if (c.t == 0) {
-              KVC_TR(m_q, ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, abort_word));
+              ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, ctl);
               if (pass == mine) cur_slot = qr.i;
               else if (ok) mbar_arrive(bar_qfree(qr.i));
             }
-            if (pass == mine) KVC_TR(m_ko, if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word));
-            else KVC_TR(m_kx, if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, abort_word));
+            if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, ctl);
             if (ok && pass != mine) mbar_arrive(bar_kempty(kr.i));
             if (pass == mine) {
               const int buf = pass * 2 + tb.i;
-              KVC_TR(m_t, if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), abort_word));
-              KVC_TR_DECL(m_i0 = KVC_TR_NOW());
+              if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), ctl);
               if (ok) {
                 tc_fence_after();
                 const uint64_t dq0 = umma_desc(sbase + SL::kQ + cur_slot * SL::kTileBytes);
@@ -684,7 +695,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 tb.next(2);
                 if (nt < 2) ++nt;
               }
-              KVC_TR_SINCE(m_i, m_i0);
             }
             if (c.t == 0) qr.next(kQSlots);
             kr.next(SL::kStages);
@@ -692,8 +702,11 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           c.advance(P);
         }
       }
-      KVC_TR_PUT(3 + 6 * mine, m_q); KVC_TR_PUT(4 + 6 * mine, m_ko); KVC_TR_PUT(5 + 6 * mine, m_kx);
-      KVC_TR_PUT(6 + 6 * mine, m_t); KVC_TR_PUT(7 + 6 * mine, m_i); KVC_TR_PUT(8 + 6 * mine, KVC_TR_NOW() - m_s);
+      // no MMA may be in flight when the TMEM columns and the shared memory are given back
+      if (nt > 0) {
+        tc_commit(bar_mma_done(mine));
+        mbar_wait_issued(bar_mma_done(mine), 0u, ctl);
+      }
     }
   } else if (warp == 3) {
     // ============================== statistics exchange ========================================
@@ -704,7 +717,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     // Lane i owns rows 4i .. 4i+3; a record of 128 rows is 64 float4, two per lane.
     const int n_groups = P.U * P.NG;
     int gi = blockIdx.x, un = blockIdx.x;             // next group / next unit of this CTA
-    bool ok = true;
+    bool ok = my_runs > 0;
     while (ok && (gi < n_groups || un < P.U)) {
       const bool take_group = gi < n_groups && (un >= P.U || gi <= (un + 1) * P.NG - 1);
       const int* counter = take_group ? P.group_counter + gi : P.unit_counter + un;
@@ -720,10 +733,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         uint32_t spins = 0;
         while (ld_acquire_s32(counter) != target) {
           __nanosleep(200);
-          if ((++spins & 63u) == 0) {
-            if (*abort_word) { ok = false; break; }
-            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_word = 1; ok = false; break; }
-          }
+          if ((++spins & 63u) == 0 && give_up(ctl, t0)) { ok = false; break; }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -734,18 +744,22 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         const int u = gi / P.NG, g = gi - u * P.NG;
         const int members = target + 1;
         const float4* src = P.partial + ((long long)u * P.RPU + g * kGroupRuns) * 64 + 2 * lane;
-        float4 v[2 * kGroupRuns];
+        // four records in flight at a time (this warp runs on a small register budget)
+#pragma unroll 1
+        for (int r0 = 0; r0 < members; r0 += 4) {
+          float4 v[8];
 #pragma unroll
-        for (int r = 0; r < kGroupRuns; ++r) {
-          if (r < members) { v[2 * r] = __ldcg(src + r * 64); v[2 * r + 1] = __ldcg(src + r * 64 + 1); }
-        }
+          for (int r = 0; r < 4; ++r) {
+            if (r0 + r < members) { v[2 * r] = __ldcg(src + (r0 + r) * 64); v[2 * r + 1] = __ldcg(src + (r0 + r) * 64 + 1); }
+          }
 #pragma unroll
-        for (int r = 0; r < kGroupRuns; ++r) {
-          if (r < members) {
-            combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
-            combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
-            combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
-            combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
+          for (int r = 0; r < 4; ++r) {
+            if (r0 + r < members) {
+              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
+              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
+              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
+              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
+            }
           }
         }
         float4* dst = P.group_partial + (long long)gi * 64 + 2 * lane;
@@ -759,7 +773,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         gi += P.grid;
       } else {
         const float4* src = P.group_partial + (long long)un * P.NG * 64 + 2 * lane;
-#pragma unroll 4
+#pragma unroll 2
         for (int r = 0; r < P.NG; ++r) {
           const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
           combine(lo.x, lo.y, v0.x, v0.y);
@@ -786,7 +800,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
 
     int n1 = 0;
-    KVC_TR_DECL(e_t = 0, e_c = 0, e_b = 0, e_s = KVC_TR_NOW());
     float mref = -INFINITY, lsum = 0.f;               // sum over the run so far of 2^(logit - mref)
     float row_ref = 0.f;                              // the row's reference exponent for the pushed sum
     bool ok = true;
@@ -829,38 +842,41 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       const bool row_used = row < c.rows(P);
       if (c.t == 0 && half == 0) row_ref = __ldg(P.ref + (long long)c.u * kRows + row);   // used at the run's end
       const int buf = n1 & 1;
-      KVC_TR(e_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), abort_word));
-      tc_fence_after();
-      const long long c0 = (long long)tile * kTile + half * 64;
-      const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;       // no masking anywhere in the tile
-      const uint32_t taddr = lane_addr + (uint32_t)buf * kTile + half * 64;
+      // (the TMEM loads below are warp-wide instructions: the decision has to be the warp's)
+      ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_tfull(buf), (uint32_t)((n1 >> 1) & 1), ctl));
       ++n1;
-      if (full) {
-        uint32_t ra[32], rb[32];
-        tc_ld32_nowait(taddr, ra);
-        tc_ld32_nowait(taddr + 32, rb);
-        tc_wait_ld(ra);
-        tc_wait_ld(rb);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tempty(buf));    // the accumulator is in registers now
-        KVC_TR(e_c, if (ok && row_used) { fast_chunk(ra); fast_chunk(rb); });
-      } else {
-        float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
-        p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
-        if (ok && row_used) { mref = m2; lsum = l2; }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tempty(buf));
+      if (ok) {
+        tc_fence_after();
+        const long long c0 = (long long)tile * kTile + half * 64;
+        const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;       // no masking anywhere in the tile
+        const uint32_t taddr = lane_addr + (uint32_t)buf * kTile + half * 64;
+        if (full) {
+          uint32_t ra[32], rb[32];
+          tc_ld32_nowait(taddr, ra);
+          tc_ld32_nowait(taddr + 32, rb);
+          tc_wait_ld(ra);
+          tc_wait_ld(rb);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty(buf));    // the accumulator is in registers now
+          if (row_used) { fast_chunk(ra); fast_chunk(rb); }
+        } else {
+          float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
+          p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
+          if (row_used) { mref = m2; lsum = l2; }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty(buf));
+        }
       }
       if (run_ends) {
         // the two halves of every row meet through shared memory; the lower half's warps write
         // the run's record and report it to the statistics warp
         if (half == 1) *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
-        KVC_TR(e_b, named_bar(3, 256));
+        named_bar(3, 256);
         const float2 other = *stage;
-        KVC_TR(e_b, named_bar(3, 256));                 // the stage may be written again
-        if (half == 0) {
+        named_bar(3, 256);                                // the stage may be written again
+        if (half == 0 && ok && c.u != P.withhold_unit) {
           float M = row_used ? mref : -INFINITY, Ls = row_used ? lsum : 0.f;
           combine(M, Ls, other.x, other.y);
           reinterpret_cast<float2*>(P.partial)[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
@@ -887,7 +903,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         mref = -INFINITY; lsum = 0.f;
       }
     }
-    if (threadIdx.x == 256) { KVC_TR_PUT(15, e_t); KVC_TR_PUT(16, e_c); KVC_TR_PUT(17, KVC_TR_NOW() - e_s); KVC_TR_PUT(22, e_b); }
   } else {
     // ============================== pass-2 epilogue ============================================
     const int quarter = warp & 3;
@@ -897,7 +912,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
     int n2 = 0;
     bool ok = true;
-    KVC_TR_DECL(f_l = 0, f_t = 0, f_c = 0, f_s = KVC_TR_NOW());
 
     Cursor cu;
     cu.init(P);
@@ -920,14 +934,13 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         // complete then).  If a run's sum did not fit, the folded
         // records decide (the value is its own flag).
         float lse = 0.f;
-        KVC_TR_DECL(f_l0 = KVC_TR_NOW());
         if (ok && trow < rows_u) {
           bool pushed = false;
           {
             if (early_u != cu.u) { early_word = 0ull; early_ref = __ldg(P.ref + (long long)cu.u * kRows + trow); }
             unsigned long long word = early_word;
             if ((unsigned int)(word >> 56) != (unsigned int)P.RPU)
-              word = poll_acc_slow(P.acc + (long long)cu.u * kRows + trow, (unsigned int)P.RPU, abort_word);
+              word = poll_acc_slow(P.acc + (long long)cu.u * kRows + trow, (unsigned int)P.RPU, ctl);
             const unsigned long long sum = word & kAccSumMask;
             if (((word >> 48) & 0xffull) == 0 && sum != 0) {
               lse = early_ref + lg2((float)sum) - (float)kAccFracBits;
@@ -937,7 +950,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           if (!pushed) {
             const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
             uint32_t bits = ld_relaxed_u32(src);
-            if (bits == 0xffffffffu) bits = poll_lse_slow(src, abort_word);
+            if (bits == 0xffffffffu) bits = poll_lse_slow(src, ctl);
             lse = __uint_as_float(bits);
           }
         }
@@ -945,8 +958,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         named_bar(1, 128);                             // everyone is done with the previous unit's values
         neg_lse[trow] = (trow < rows_u) ? -lse : 0.f;
         named_bar(1, 128);
-        KVC_TR_SINCE(f_l, f_l0);
-        if (*abort_word) ok = false;
+        ok = !__any_sync(0xffffffffu, ctl->abort != 0) && ok;
       }
       if (early_u < 0 && cu.t >= P.RT - 2 && idx + (P.RT - cu.t) < my_tiles) {
         // the next run's word and reference: in flight while the rest of this run is computed
@@ -958,9 +970,10 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       }
       const int buf = 2 + (n2 & 1);
       const uint32_t tmem_col = (uint32_t)buf * kTile;
-      KVC_TR(f_t, if (ok) ok = mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), abort_word));
-      KVC_TR_DECL(f_c1 = KVC_TR_NOW());
+      // (the TMEM loads below are warp-wide instructions: the decision has to be the warp's)
+      ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_tfull(buf), (uint32_t)((n2 >> 1) & 1), ctl));
       ++n2;
+      if (!ok) continue;
       tc_fence_after();
       const long long c = (long long)tile * kTile + trow;            // this thread's token
       const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;
@@ -1017,17 +1030,15 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       }
       // one row tile: the group aggregate itself; several: this tile's part of it
       if (P.QT == 1 && P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
-      if (ok && c < P.N)
+      if (c < P.N)
         P.scores[((long long)cu.q * ((long long)P.L * P.Bt * P.Hkv) + cu.kv_unit(P)) * P.N + c] = gacc;
-      KVC_TR_SINCE(f_c, f_c1);
     }
-    if (threadIdx.x == 128) { KVC_TR_PUT(18, f_l); KVC_TR_PUT(19, f_t); KVC_TR_PUT(20, f_c); KVC_TR_PUT(21, KVC_TR_NOW() - f_s); }
   }
 
   // ---------------- teardown ----------------
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *abort_word && P.status) atomicCAS(P.status, 0, (int)KVC_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && ctl->abort && P.status) atomicCAS(P.status, 0, (int)KVC_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -1096,15 +1107,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 EncodeTiledFn encode_fn() {
   static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static std::once_flag once;
+  std::call_once(once, [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+  });
   return fn;
 }
 
@@ -1165,14 +1175,42 @@ int sm_count() {
   return sms;
 }
 
+// Test hooks (kvc_debug_score_hooks): the bound of the device-side waits and a unit whose
+// statistics are withheld.
+std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
+std::atomic<int> g_withhold_unit{-1};
+
+constexpr int kMaxDevices = 64;
+std::mutex g_launch_mutex;
+
+// The kernel's CTAs wait for one another, so all of them have to be resident at once: one per
+// SM with the opt-in amount of shared memory.  Checked once per device and instantiation (the
+// attribute is per device); KVC_ERR_UNSUPPORTED sends the caller to the CUDA-core path.
+template <int D, int W, bool M>
+kvc_status prepare_t(int grid) {
+  using SL = SmemLayout<D>;
+  static signed char state[kMaxDevices];      // 0: not looked at, 1: fits, -1: does not
+  int dev = 0;
+  KVC_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return KVC_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_launch_mutex);
+  if (state[dev] == 0) {
+    KVC_CUDA(cudaFuncSetAttribute(score_sm100_kernel<D, W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal));
+    int per_sm = 0, sms = 0;
+    KVC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_sm100_kernel<D, W, M>, kFastThreads,
+                                                           (size_t)SL::kTotal));
+    KVC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    state[dev] = (per_sm >= 1 && sms >= 1) ? 1 : -1;
+  }
+  (void)grid;                                 // grid <= SM count by construction (make_plan)
+  return state[dev] == 1 ? KVC_OK : KVC_ERR_UNSUPPORTED;
+}
+
 template <int D, int W, bool M>
 kvc_status launch_t(const FastParams& fp, int grid, cudaStream_t st) {
   using SL = SmemLayout<D>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    KVC_CUDA(cudaFuncSetAttribute(score_sm100_kernel<D, W, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal));
-    attr_set = true;
-  }
+  const kvc_status s = prepare_t<D, W, M>(grid);
+  if (s != KVC_OK) return s;
   KVC_CUDA(launch_dependent(score_sm100_kernel<D, W, M>, dim3(grid), dim3(kFastThreads), (size_t)SL::kTotal, st, fp));
   KVC_LAUNCH_CHECK("score_sm100_kernel");
   return KVC_OK;
@@ -1269,6 +1307,8 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.step_l = fp.step_u / pl.QT / P.Hkv / P.Bt;
   fp.sl2e = P.scale * kLog2eF;
   fp.agg_group = P.agg_group;
+  fp.wait_limit_ns = g_wait_limit_ns.load();
+  fp.withhold_unit = g_withhold_unit.load();
   const bool mean = P.agg_task == KVC_AGG_MEAN;
   if (P.d == 128) return mean ? launch_w<128, true>(P.w, fp, pl.grid, st) : launch_w<128, false>(P.w, fp, pl.grid, st);
   return mean ? launch_w<64, true>(P.w, fp, pl.grid, st) : launch_w<64, false>(P.w, fp, pl.grid, st);
@@ -1276,9 +1316,12 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
 
 }  // namespace kvc
 
-#ifdef KVC_SCORE_TRACE
-// Debug builds only: copies the trace counters (160 x 24 words) to the host.
-extern "C" __attribute__((visibility("default"))) int kvc_debug_dump(unsigned long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, kvc::g_score_trace, sizeof(unsigned long long) * 160 * 24);
+
+// Test hook: the bound of the scoring kernel's device-side waits (<= 0: the default of 2 s) and a
+// unit (layer, sequence, KV head, row tile in that order) whose statistics are never sent, so
+// that the waits for them expire (-1: none).  Process-wide; takes effect at the next launch.
+extern "C" __attribute__((visibility("default"))) void kvc_debug_score_hooks(int64_t wait_limit_ns,
+                                                                             int32_t withhold_unit) {
+  kvc::g_wait_limit_ns.store(wait_limit_ns > 0 ? (unsigned long long)wait_limit_ns : kvc::kDefaultWaitLimitNs);
+  kvc::g_withhold_unit.store(withhold_unit);
 }
-#endif
