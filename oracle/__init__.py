@@ -7,6 +7,7 @@ from .api import (  # noqa: F401
     AGG_MAX,
     AGG_MEAN,
     allocate,
+    allocate_floor,
     attention_rows,
     budget_from_ratio,
     build,
@@ -18,5 +19,8 @@ from .api import (  # noqa: F401
     has_openmp,
     rank,
     score_layer,
+    score_layer_vnorm,
+    select_unstructured,
     set_threads,
+    sort_kept,
 )

@@ -51,6 +51,14 @@ def _load():
     lib.oracle_attention_rows.restype = None
     lib.oracle_score_layer.argtypes = [p, p, i32, i32, i64, i32, i32, f64, i64, i32, i32, i32, p, p]
     lib.oracle_score_layer.restype = C.c_int
+    lib.oracle_score_layer_vnorm.argtypes = [p, p, p, i32, i32, i64, i32, i32, f64, i64, i32, i32, i32, p, p]
+    lib.oracle_score_layer_vnorm.restype = C.c_int
+    lib.oracle_allocate_floor.argtypes = [p, i32, i64, i64, i64, p, p]
+    lib.oracle_allocate_floor.restype = C.c_int
+    lib.oracle_select_unstructured.argtypes = [p, i32, i32, i64, i64, p, p]
+    lib.oracle_select_unstructured.restype = C.c_int
+    lib.oracle_sort_kept.argtypes = [p, i32, i64, p, p]
+    lib.oracle_sort_kept.restype = None
     lib.oracle_rank.argtypes = [p, i64, p, p]
     lib.oracle_rank.restype = C.c_int
     lib.oracle_compose.argtypes = [p, i32, i64, i32, p]
@@ -126,6 +134,23 @@ def score_layer(q, k, scale, q_pos0, agg_task=AGG_MAX, agg_group=AGG_MEAN, augme
     return S
 
 
+def score_layer_vnorm(q, k, v, scale, q_pos0, agg_task=AGG_MAX, agg_group=AGG_MEAN, augment=True,
+                      q_to_kv=None):
+    """The v-norm variant (App. A.1.3): q [Hq, w, d], k, v [Hkv, N, d] -> S [Hkv, N] float64."""
+    q, k, v = _f32(q), _f32(k), _f32(v)
+    Hq, w, d = q.shape
+    Hkv, N, d2 = k.shape
+    assert d == d2 and v.shape == k.shape
+    m = _map(q_to_kv, Hq)
+    S = np.empty((Hkv, N), dtype=np.float64)
+    rc = _load().oracle_score_layer_vnorm(_ptr(q), _ptr(k), _ptr(v), Hq, Hkv, N, d, w, float(scale),
+                                          int(q_pos0), int(agg_task), int(agg_group),
+                                          int(bool(augment)), _ptr(m), _ptr(S))
+    if rc:
+        raise RuntimeError("oracle_score_layer_vnorm failed (%d)" % rc)
+    return S
+
+
 def rank(S):
     """S [N] -> (idx [N] int32, S_sorted [N] float64): Eqs. 17-18, ties to the smaller position."""
     S = np.ascontiguousarray(S, dtype=np.float64)
@@ -169,6 +194,41 @@ def allocate(I, B):
     if rc:
         raise ValueError("oracle_allocate failed (%d)" % rc)
     return n_keep, offsets
+
+
+def allocate_floor(I, B, min_keep):
+    """Eqs. 20-22 with a per-layer minimum: I [L, N] -> (n_keep [L], offsets [L+1])."""
+    I = np.ascontiguousarray(I, dtype=np.float64)
+    L, N = I.shape
+    n_keep = np.empty(L, dtype=np.int32)
+    offsets = np.empty(L + 1, dtype=np.int64)
+    rc = _load().oracle_allocate_floor(_ptr(I), L, N, int(B), int(min_keep), _ptr(n_keep), _ptr(offsets))
+    if rc:
+        raise ValueError("oracle_allocate_floor failed (%d)" % rc)
+    return n_keep, offsets
+
+
+def select_unstructured(S, B):
+    """App. A.2: S [L, Hkv, N] -> (n_keep [L, Hkv] int32, offsets [L*Hkv+1] int64): the B best
+    entries of the pool over (layer, head, position)."""
+    S = np.ascontiguousarray(S, dtype=np.float64)
+    L, Hkv, N = S.shape
+    n_keep = np.empty(L * Hkv, dtype=np.int32)
+    offsets = np.empty(L * Hkv + 1, dtype=np.int64)
+    rc = _load().oracle_select_unstructured(_ptr(S), L, Hkv, N, int(B), _ptr(n_keep), _ptr(offsets))
+    if rc:
+        raise ValueError("oracle_select_unstructured failed (%d)" % rc)
+    return n_keep.reshape(L, Hkv), offsets
+
+
+def sort_kept(idx, n_keep):
+    """idx [Hkv, N], n_keep [Hkv] -> idx with every head's first n_keep[h] positions ascending."""
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    Hkv, N = idx.shape
+    nk = np.ascontiguousarray(np.broadcast_to(np.asarray(n_keep, dtype=np.int32), (Hkv,)))
+    out = np.empty_like(idx)
+    _load().oracle_sort_kept(_ptr(idx), Hkv, N, _ptr(nk), _ptr(out))
+    return out
 
 
 def gather_layer(src, idx, n_keep):

@@ -110,10 +110,10 @@ void oracle_attention_rows(const float* q, const float* k, int64_t N, int32_t d,
  * S[h, c]        = S_group[h, c] + (1/Hkv) sum_i S_group[i, c]       (Eq. 16)
  * Returns 0, or -1 on allocation failure / a KV head without query heads.
  */
-int oracle_score_layer(const float* q, const float* k, int32_t Hq, int32_t Hkv,
-                       int64_t N, int32_t d, int32_t w, double scale,
-                       int64_t q_pos0, int32_t agg_task, int32_t agg_group,
-                       int32_t augment, const int32_t* q_to_kv, double* S) {
+static int score_layer_impl(const float* q, const float* k, const float* v, int32_t Hq,
+                            int32_t Hkv, int64_t N, int32_t d, int32_t w, double scale,
+                            int64_t q_pos0, int32_t agg_task, int32_t agg_group,
+                            int32_t augment, const int32_t* q_to_kv, double* S) {
   int32_t G = Hq / Hkv;
   double* S_task = (double*)malloc(sizeof(double) * (size_t)Hq * (size_t)N);
   if (!S_task) return -1;
@@ -135,6 +135,19 @@ int oracle_score_layer(const float* q, const float* k, int32_t Hq, int32_t Hkv,
     }
     oracle_attention_rows(q + (int64_t)j * w * d, k + (int64_t)h * N * d, N, d, w,
                           scale, q_pos0, A);
+    if (v) {
+      /* App. A.1.3, the v-norm variant: every entry of A is multiplied by the Euclidean
+         norm of the value row of its token (in the KV head this query head reads). */
+      for (int64_t c = 0; c < N; ++c) {
+        double nn = 0.0;
+        for (int32_t t = 0; t < d; ++t) {
+          double x = (double)v[((int64_t)h * N + c) * d + t];
+          nn += x * x;
+        }
+        nn = sqrt(nn);
+        for (int32_t m = 0; m < w; ++m) A[(int64_t)m * N + c] *= nn;
+      }
+    }
     for (int64_t c = 0; c < N; ++c) {
       double acc = (agg_task == ORACLE_AGG_MAX) ? -INFINITY : 0.0;
       for (int32_t m = 0; m < w; ++m) {
@@ -189,6 +202,28 @@ int oracle_score_layer(const float* q, const float* k, int32_t Hq, int32_t Hkv,
     }
   }
   return 0;
+}
+
+int oracle_score_layer(const float* q, const float* k, int32_t Hq, int32_t Hkv,
+                       int64_t N, int32_t d, int32_t w, double scale,
+                       int64_t q_pos0, int32_t agg_task, int32_t agg_group,
+                       int32_t augment, const int32_t* q_to_kv, double* S) {
+  return score_layer_impl(q, k, NULL, Hq, Hkv, N, d, w, scale, q_pos0, agg_task, agg_group,
+                          augment, q_to_kv, S);
+}
+
+/*
+ * The v-norm variant of App. A.1.3 ("Effect of Value Norms on Token Scores"): the weighted
+ * attention matrix A^(w)[m, c] = A[m, c] * ||v_c|| replaces A in Eqs. (14)-(16).
+ * v [Hkv, N, d]: the value rows; the norm is the Euclidean norm over the d entries of a row.
+ */
+int oracle_score_layer_vnorm(const float* q, const float* k, const float* v, int32_t Hq,
+                             int32_t Hkv, int64_t N, int32_t d, int32_t w, double scale,
+                             int64_t q_pos0, int32_t agg_task, int32_t agg_group,
+                             int32_t augment, const int32_t* q_to_kv, double* S) {
+  if (!v) return -1;
+  return score_layer_impl(q, k, v, Hq, Hkv, N, d, w, scale, q_pos0, agg_task, agg_group,
+                          augment, q_to_kv, S);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -331,6 +366,110 @@ int oracle_allocate(const double* I, int32_t L, int64_t N, int64_t B, int32_t* n
   offsets[0] = 0;
   for (int32_t l = 0; l < L; ++l) offsets[l + 1] = offsets[l] + n_keep[l];
   return 0;
+}
+
+/*
+ * Eqs. (20)-(22) with a per-layer minimum (an option the paper does not have: nothing in
+ * Sec. 3.3 keeps a layer from getting no slot at all).  Every layer first keeps its
+ * min_keep best composite tokens; the remaining B - L * min_keep slots go to the best of
+ * all other pooled entries under the same total order.  min_keep = 0 is oracle_allocate.
+ */
+int oracle_allocate_floor(const double* I, int32_t L, int64_t N, int64_t B, int64_t min_keep,
+                          int32_t* n_keep, int64_t* offsets) {
+  if (min_keep < 0 || min_keep > N || (int64_t)L * min_keep > B) return -2;
+  int64_t rest = N - min_keep;
+  int64_t total = (int64_t)L * rest;
+  int64_t Brest = B - (int64_t)L * min_keep;
+  if (Brest > total) return -2;
+  pool_item* P = (pool_item*)malloc(sizeof(pool_item) * (size_t)(total > 0 ? total : 1));
+  if (!P) return -1;
+  for (int32_t l = 0; l < L; ++l)
+    for (int64_t kk = min_keep; kk < N; ++kk) {
+      pool_item* p = &P[(int64_t)l * rest + (kk - min_keep)];
+      p->v = I[(int64_t)l * N + kk];
+      p->l = l;
+      p->k = kk;
+    }
+  qsort(P, (size_t)total, sizeof(pool_item), pool_cmp);
+  for (int32_t l = 0; l < L; ++l) n_keep[l] = (int32_t)min_keep;
+  for (int64_t i = 0; i < Brest; ++i) n_keep[P[i].l] += 1;
+  free(P);
+  offsets[0] = 0;
+  for (int32_t l = 0; l < L; ++l) offsets[l + 1] = offsets[l] + n_keep[l];
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* App. A.2: the unstructured variant                                          */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+  double v;
+  int32_t l, h;
+  int64_t c;
+} entry_item;
+
+/* order: score descending, then layer, head, position ascending */
+static int entry_cmp(const void* a, const void* b) {
+  const entry_item* x = (const entry_item*)a;
+  const entry_item* y = (const entry_item*)b;
+  if (x->v > y->v) return -1;
+  if (x->v < y->v) return 1;
+  if (x->l != y->l) return x->l < y->l ? -1 : 1;
+  if (x->h != y->h) return x->h < y->h ? -1 : 1;
+  if (x->c < y->c) return -1;
+  if (x->c > y->c) return 1;
+  return 0;
+}
+
+/*
+ * App. A.2 ("Discussion on unstructured eviction methods"): the final aggregation over the
+ * heads (Eq. 19) is left out and every head keeps its own tokens.  All entries S[l, h, c]
+ * of one sequence form one pool; the B best are kept (ties: layer, head, position
+ * ascending); n_keep[l, h] = how many of them lie in head h of layer l -- those are the
+ * head's n_keep[l, h] best tokens, i.e. the first n_keep[l, h] entries of its ranking
+ * (Eq. 17).  offsets = exclusive prefix sum over (l, h) in that order.
+ *   S [L, Hkv, N] -> n_keep [L * Hkv], offsets [L * Hkv + 1].
+ */
+int oracle_select_unstructured(const double* S, int32_t L, int32_t Hkv, int64_t N, int64_t B,
+                               int32_t* n_keep, int64_t* offsets) {
+  int64_t total = (int64_t)L * Hkv * N;
+  if (B < 0 || B > total) return -2;
+  entry_item* P = (entry_item*)malloc(sizeof(entry_item) * (size_t)(total > 0 ? total : 1));
+  if (!P) return -1;
+  for (int32_t l = 0; l < L; ++l)
+    for (int32_t h = 0; h < Hkv; ++h)
+      for (int64_t c = 0; c < N; ++c) {
+        entry_item* p = &P[((int64_t)l * Hkv + h) * N + c];
+        p->v = S[((int64_t)l * Hkv + h) * N + c];
+        p->l = l;
+        p->h = h;
+        p->c = c;
+      }
+  qsort(P, (size_t)total, sizeof(entry_item), entry_cmp);
+  for (int32_t r = 0; r < L * Hkv; ++r) n_keep[r] = 0;
+  for (int64_t i = 0; i < B; ++i) n_keep[P[i].l * Hkv + P[i].h] += 1;
+  free(P);
+  offsets[0] = 0;
+  for (int32_t r = 0; r < L * Hkv; ++r) offsets[r + 1] = offsets[r] + n_keep[r];
+  return 0;
+}
+
+static int int32_cmp(const void* a, const void* b) {
+  int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+  return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+/*
+ * Output order option: the kept tokens of a head in their original order.
+ * idx [Hkv, N] (Eq. 17), n_keep[h] kept per head -> out [Hkv, N]: out[h, :n_keep[h]] are the
+ * positions idx[h, :n_keep[h]] in ascending order; the rest of the row is copied unchanged.
+ */
+void oracle_sort_kept(const int32_t* idx, int32_t Hkv, int64_t N, const int32_t* n_keep,
+                      int32_t* out) {
+  memcpy(out, idx, sizeof(int32_t) * (size_t)Hkv * (size_t)N);
+  for (int32_t h = 0; h < Hkv; ++h)
+    qsort(out + (int64_t)h * N, (size_t)n_keep[h], sizeof(int32_t), int32_cmp);
 }
 
 /* ------------------------------------------------------------------------- */
