@@ -88,6 +88,21 @@ typedef struct {
                                 Eq. 15; then Hq % Hkv must be 0).  Every KV head needs >= 1 member. */
   int64_t q_stride[3];
   int64_t kv_stride[3];
+  /* Options beyond the paper's default pipeline; kvc_desc_init sets all of them to 0. */
+  int32_t value_norm;          /* 1: the v-norm variant of App. A.1.3 -- every attention weight A[m, c] is
+                                  multiplied by the Euclidean norm of token c's value row (in the KV head the
+                                  query head reads) before Eq. 14.  Used by kvc_compress and
+                                  kvc_compress_unstructured (which have V); kvc_score refuses it, use
+                                  kvc_score_weighted. */
+  int32_t min_keep_per_layer;  /* per-layer minimum m for Eq. 22 (the paper has none: a layer may get no
+                                  slot): every layer first keeps its m best composite tokens, the other
+                                  budget - L * m slots are handed out as in Eqs. 20-22 among the rest.
+                                  0 <= m <= N and L * m <= budget.  Used by kvc_allocate, kvc_compress. */
+  int32_t keep_position_order; /* 1: the rows of a head in K', V' come in ascending original position
+                                  instead of descending score (the kept set is the same).  Used by
+                                  kvc_compress and kvc_compress_unstructured; staged callers apply
+                                  kvc_order_kept to idx before kvc_gather. */
+  int32_t reserved_;           /* must be 0 */
 } kvc_desc;
 
 /* Fill *desc with the paper's defaults for the given shape (dense strides, q_pos0 = N - w,
@@ -101,7 +116,8 @@ KVC_API void kvc_desc_init(kvc_desc* desc, int32_t n_layers, int32_t batch, int3
  * behave as in exact arithmetic.  Returns -1 on a bad descriptor or r_target outside [0, 1]. */
 KVC_API int64_t kvc_budget_from_ratio(const kvc_desc* desc, double r_target);
 
-/* Bytes of scratch any entry point below may need for this problem and budget (host call). */
+/* Bytes of scratch any entry point below may need for this problem (with the options set in desc)
+ * and budget (host call). */
 KVC_API kvc_status kvc_workspace_size(const kvc_desc* desc, int64_t budget, size_t* bytes);
 
 /*
@@ -124,6 +140,18 @@ KVC_API kvc_status kvc_score(const kvc_desc* desc, const void* const* q, const v
 /* Byte offset, inside the workspace handed to kvc_score, of the int32 device status word that call
  * writes (host call; depends on the problem only). */
 KVC_API kvc_status kvc_score_status_offset(const kvc_desc* desc, size_t* offset);
+
+/*
+ * kvc_score with value-norm weighting (App. A.1.3 "Effect of Value Norms on Token Scores", the
+ * v-norm variant): A^(w)[m, c] = A[m, c] * ||v[kv(j), c]||_2 takes the place of A in Eqs. 14-16.
+ * v: HOST array of n_layers device pointers, laid out like k.  The norm of a row is taken in fp32
+ * over its head_dim entries.  Because the weight depends on (KV head, token) only and the pooling
+ * operators are positively homogeneous, the weighting is applied to the group aggregate of Eq. 15.
+ * Everything else as kvc_score (same workspace, same status word); desc->value_norm is ignored.
+ */
+KVC_API kvc_status kvc_score_weighted(const kvc_desc* desc, const void* const* q, const void* const* k,
+                              const void* const* v, float* scores, void* workspace,
+                              size_t workspace_bytes, void* stream);
 
 /*
  * Ranking and composite tokens (Sec. 3.3).  For every (l, b, h):
@@ -150,6 +178,15 @@ KVC_API kvc_status kvc_compose(const kvc_desc* desc, const float* scores, int32_
 KVC_API kvc_status kvc_allocate(const kvc_desc* desc, const float* composite, int64_t budget,
                         int32_t* n_keep, int64_t* offsets, void* workspace,
                         size_t workspace_bytes, void* stream);
+
+/*
+ * Output order option (the paper keeps idx[:N_l], i.e. descending score, Eq. 23): rewrites, in
+ * place, the first n_keep[b, l] entries of every idx[l, b, h, :] in ascending position; the rest
+ * of each row is left as it is.  A later kvc_gather then writes each head's rows of K', V' in
+ * their original order.  n_keep: [batch, L] (device).  Scratch: kvc_workspace_size bytes.
+ */
+KVC_API kvc_status kvc_order_kept(const kvc_desc* desc, int32_t* idx, const int32_t* n_keep,
+                          void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * kvc_allocate without a workspace argument (the paper has no counterpart to this entry point; it
@@ -204,6 +241,35 @@ KVC_API kvc_status kvc_compress(const kvc_desc* desc, const void* const* q, cons
                         int32_t* n_keep, int64_t* offsets, int32_t* idx_out, float* scores_out,
                         float* composite_out, int32_t* device_status, void* workspace,
                         size_t workspace_bytes, void* stream);
+
+/*
+ * The unstructured variant (App. A.2 "Discussion on unstructured eviction methods"): the
+ * aggregation over the heads (Eq. 19) is left out and every head keeps its own tokens.  Per
+ * sequence, all entries scores[l, b, h, c] form one pool; the `budget_entries` best are kept (ties:
+ * layer, head, position ascending -- the structured budget of Eq. 21 corresponds to
+ * budget_entries = B_total * Hkv); n_keep[b, l, h] = how many of them lie in head h of layer l,
+ * which are the first n_keep[b, l, h] entries of idx[l, b, h, :].
+ *
+ * kvc_select_unstructured: ranking (Eq. 17) and the global selection.
+ *   idx:     [L, batch, Hkv, N] int32            n_keep: [batch, L, Hkv] int32
+ *   offsets: [batch, L * Hkv + 1] int64, exclusive prefix sum of n_keep over (l, h)
+ * kvc_gather_unstructured: k_out, v_out [batch, budget_entries * d]; head (l, h) of sequence b
+ *   starts at element offsets[b, l * Hkv + h] * d and is a dense [n_keep[b, l, h], d] tensor (a
+ *   ragged cache: heads of a layer differ in length).
+ * kvc_compress_unstructured: score (with desc->value_norm if set) + select + (position order if
+ *   set) + gather, stream-ordered.  L * Hkv <= 2048.  0 <= budget_entries <= L * Hkv * N.
+ */
+KVC_API kvc_status kvc_select_unstructured(const kvc_desc* desc, const float* scores, int64_t budget_entries,
+                                   int32_t* idx, int32_t* n_keep, int64_t* offsets, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+KVC_API kvc_status kvc_gather_unstructured(const kvc_desc* desc, const void* const* k, const void* const* v,
+                                   const int32_t* idx, const int32_t* n_keep, const int64_t* offsets,
+                                   int64_t budget_entries, void* k_out, void* v_out, void* stream);
+KVC_API kvc_status kvc_compress_unstructured(const kvc_desc* desc, const void* const* q, const void* const* k,
+                                     const void* const* v, int64_t budget_entries, void* k_out,
+                                     void* v_out, int32_t* n_keep, int64_t* offsets, int32_t* idx_out,
+                                     float* scores_out, int32_t* device_status, void* workspace,
+                                     size_t workspace_bytes, void* stream);
 
 /* Message of the last error returned on this thread (static storage; never NULL). */
 KVC_API const char* kvc_last_error(void);

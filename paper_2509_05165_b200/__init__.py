@@ -16,13 +16,18 @@ from .binding import (  # noqa: F401
     kvc_budget_from_ratio,
     kvc_compose,
     kvc_compress,
+    kvc_compress_unstructured,
     kvc_desc_init,
     kvc_gather,
+    kvc_gather_unstructured,
+    kvc_order_kept,
     kvc_last_error,
     kvc_launch_count,
     kvc_debug_score_hooks,
     kvc_score,
     kvc_score_status_offset,
+    kvc_score_weighted,
+    kvc_select_unstructured,
     kvc_version,
     kvc_workspace_size,
     library_path,

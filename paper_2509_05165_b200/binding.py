@@ -32,6 +32,8 @@ class KvcDesc(C.Structure):
         ("agg_task", C.c_int32), ("agg_group", C.c_int32), ("agg_head", C.c_int32),
         ("augment_head_mean", C.c_int32), ("q_to_kv", C.POINTER(C.c_int32)),
         ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3),
+        ("value_norm", C.c_int32), ("min_keep_per_layer", C.c_int32), ("keep_position_order", C.c_int32),
+        ("reserved_", C.c_int32),
     ]
 
 
@@ -70,6 +72,16 @@ def _load():
     lib.kvc_score_status_offset.restype = C.c_int
     lib.kvc_debug_score_hooks.argtypes = [i64, i32]
     lib.kvc_debug_score_hooks.restype = None
+    lib.kvc_score_weighted.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+    lib.kvc_score_weighted.restype = C.c_int
+    lib.kvc_order_kept.argtypes = [dp, vp, vp, vp, sz, vp]
+    lib.kvc_order_kept.restype = C.c_int
+    lib.kvc_select_unstructured.argtypes = [dp, vp, i64, vp, vp, vp, vp, sz, vp]
+    lib.kvc_select_unstructured.restype = C.c_int
+    lib.kvc_gather_unstructured.argtypes = [dp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.kvc_gather_unstructured.restype = C.c_int
+    lib.kvc_compress_unstructured.argtypes = [dp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.kvc_compress_unstructured.restype = C.c_int
     lib.kvc_compose.argtypes = [dp, vp, vp, vp, vp, sz, vp]
     lib.kvc_compose.restype = C.c_int
     lib.kvc_allocate.argtypes = [dp, vp, i64, vp, vp, vp, sz, vp]
@@ -141,6 +153,13 @@ def kvc_score(desc, q: Sequence[torch.Tensor], k: Sequence[torch.Tensor], scores
                              _stream(stream)))
 
 
+def kvc_score_weighted(desc, q, k, v, scores: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    """``kvc_score`` with the attention weights multiplied by the tokens' value norms (v-norm variant)."""
+    wp, wb = _ws(workspace)
+    _check(_load().kvc_score_weighted(C.byref(desc), _ptr_array(q), _ptr_array(k), _ptr_array(v), _dptr(scores),
+                                      wp, wb, _stream(stream)))
+
+
 def kvc_score_status_offset(desc: KvcDesc) -> int:
     """Byte offset, in the workspace given to ``kvc_score``, of that call's int32 device status."""
     out = C.c_size_t(0)
@@ -171,6 +190,32 @@ def kvc_allocate_static(desc, composite, budget, n_keep, offsets, stream=None) -
     inside the library (batch <= 64).  Calls that overlap on the GPU share that array and race."""
     _check(_load().kvc_allocate_static(C.byref(desc), _dptr(composite), int(budget), _dptr(n_keep),
                                        _dptr(offsets), _stream(stream)))
+
+
+def kvc_order_kept(desc, idx, n_keep, workspace, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_load().kvc_order_kept(C.byref(desc), _dptr(idx), _dptr(n_keep), wp, wb, _stream(stream)))
+
+
+def kvc_select_unstructured(desc, scores, budget_entries, idx, n_keep, offsets, workspace, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_load().kvc_select_unstructured(C.byref(desc), _dptr(scores), int(budget_entries), _dptr(idx),
+                                           _dptr(n_keep), _dptr(offsets), wp, wb, _stream(stream)))
+
+
+def kvc_gather_unstructured(desc, k, v, idx, n_keep, offsets, budget_entries, k_out, v_out, stream=None) -> None:
+    _check(_load().kvc_gather_unstructured(C.byref(desc), _ptr_array(k), _ptr_array(v), _dptr(idx), _dptr(n_keep),
+                                           _dptr(offsets), int(budget_entries), _dptr(k_out), _dptr(v_out),
+                                           _stream(stream)))
+
+
+def kvc_compress_unstructured(desc, q, k, v, budget_entries, k_out, v_out, n_keep, offsets, idx_out=None,
+                              scores_out=None, device_status=None, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_load().kvc_compress_unstructured(C.byref(desc), _ptr_array(q), _ptr_array(k), _ptr_array(v),
+                                             int(budget_entries), _dptr(k_out), _dptr(v_out), _dptr(n_keep),
+                                             _dptr(offsets), _dptr(idx_out), _dptr(scores_out),
+                                             _dptr(device_status), wp, wb, _stream(stream)))
 
 
 def kvc_gather(desc, k, v, idx, n_keep, offsets, budget, k_out, v_out, stream=None) -> None:

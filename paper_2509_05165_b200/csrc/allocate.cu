@@ -9,6 +9,10 @@
 // four histogram passes over the pool (each CTA re-derives the prefix chosen so far from the
 // previous passes' global histograms), then one small kernel does the per-layer binary searches
 // and the tie hand-out.
+//
+// The rows of the pool are the layers (Eqs. 20-22) or, for the unstructured variant of App. A.2,
+// the (layer, head) pairs with the heads' sorted scores as rows.  With a per-layer minimum m the
+// first m entries of every row are kept outright and stay out of the pool.
 #include "kvc_internal.cuh"
 
 namespace kvc {
@@ -20,6 +24,13 @@ constexpr int kItemsPerThread = 16;
 
 // Select state after `passes` completed passes: the key prefix (high bits) and the rank that is
 // still to be located inside that prefix bucket.  rank is 1-based among ascending keys.
+// Where row r of sequence b starts: rows are layers of composite [L, Bt, N] (heads_per_row = 1) or
+// (layer, head) pairs of sorted scores [L, Bt, Hkv, N] (heads_per_row = Hkv).
+__device__ __forceinline__ long long row_start(long long r, int b, int Bt, int hpr, long long N) {
+  const long long l = r / hpr, h = r - l * hpr;
+  return ((l * Bt + b) * hpr + h) * N;
+}
+
 struct SelectState {
   uint32_t prefix;
   unsigned long long rank;
@@ -78,9 +89,11 @@ select_clear_kernel(unsigned int* __restrict__ hist) {
   hist[(size_t)blockIdx.x * 4 * kRadix + threadIdx.x] = 0u;
 }
 
+// R rows per sequence, each of N entries of which the first `floor` are out of the pool; `budget`
+// is what is left to hand out among the others.
 __global__ void __launch_bounds__(kHistThreads)
 select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict__ hist, int pass,
-                   int L, int Bt, long long N, long long budget) {
+                   int R, int Bt, int hpr, long long N, long long floor, long long budget) {
   __shared__ unsigned int sh[kRadix];
   __shared__ unsigned long long scratch[16];
   grid_dependency_wait();
@@ -92,21 +105,22 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
   const uint32_t prefix = st.prefix;
   const int shift = 24 - 8 * pass;
   const uint32_t hi_mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
-  const long long total = (long long)L * N;
+  const long long M = N - floor;                       // pooled entries per row
+  const long long total = (long long)R * M;
   const long long tile = (long long)kHistThreads * kItemsPerThread;
   for (long long t0 = (long long)blockIdx.x * tile; t0 < total; t0 += (long long)gridDim.x * tile) {
-    // pooled index -> (layer, position) once per tile, then by steps of the block width
+    // pooled index -> (row, position) once per tile, then by steps of the block width
     long long i = t0 + threadIdx.x;
-    long long l = i / N, kk = i - l * N;
+    long long r = i / M, kk = i - r * M;
 #pragma unroll 4
     for (int it = 0; it < kItemsPerThread; ++it) {
       if (i < total) {
-        const uint32_t key = score_to_key(composite[(l * Bt + b) * N + kk]);
+        const uint32_t key = score_to_key(composite[row_start(r, b, Bt, hpr, N) + floor + kk]);
         if ((key & hi_mask) == prefix) atomicAdd(&sh[(key >> shift) & 0xffu], 1u);
       }
       i += kHistThreads;
       kk += kHistThreads;
-      while (kk >= N) { kk -= N; ++l; }
+      while (kk >= M) { kk -= M; ++r; }
     }
   }
   __syncthreads();
@@ -147,41 +161,43 @@ __device__ inline void count_layer_warp(const float* __restrict__ row, long long
   *ge = res[1];
 }
 
+// `budget` is again what is left to hand out beyond the rows' first `floor` entries.
 __global__ void __launch_bounds__(1024)
 select_finish_kernel(const float* __restrict__ composite,
-                     const unsigned int* __restrict__ hist, int L, int Bt, long long N,
-                     long long budget, int32_t* __restrict__ n_keep,
+                     const unsigned int* __restrict__ hist, int R, int Bt, int hpr, long long N,
+                     long long floor, long long budget, int32_t* __restrict__ n_keep,
                      long long* __restrict__ offsets) {
-  __shared__ long long s_gt[KVC_MAX_LAYERS];
-  __shared__ long long s_ge[KVC_MAX_LAYERS];
+  extern __shared__ long long s_cnt[];               // [R] strictly better than T, [R] at least as good
+  long long* s_gt = s_cnt;
+  long long* s_ge = s_cnt + R;
   __shared__ unsigned long long scratch[16];
   grid_dependency_wait();
   const int b = blockIdx.x;
   const SelectState st = derive_state(hist + (size_t)b * 4 * kRadix, 4, (unsigned long long)budget, scratch);
   const uint32_t T = st.prefix;
   const int warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  for (int l = warp; l < L; l += n_warps) {
+  for (int r = warp; r < R; r += n_warps) {
     long long gt = 0, ge = 0;
-    if (budget > 0) count_layer_warp(composite + ((long long)l * Bt + b) * N, N, T, &gt, &ge);
-    if ((threadIdx.x & 31) == 0) { s_gt[l] = gt; s_ge[l] = ge; }
+    if (budget > 0) count_layer_warp(composite + row_start(r, b, Bt, hpr, N) + floor, N - floor, T, &gt, &ge);
+    if ((threadIdx.x & 31) == 0) { s_gt[r] = gt; s_ge[r] = ge; }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     long long used = 0;
-    for (int l = 0; l < L; ++l) used += s_gt[l];
-    long long rem = budget - used;     // entries equal to T still to hand out, in layer order
+    for (int r = 0; r < R; ++r) used += s_gt[r];
+    long long rem = budget - used;     // entries equal to T still to hand out, in row order
     long long off = 0;
-    for (int l = 0; l < L; ++l) {
-      long long take = s_ge[l] - s_gt[l];
+    for (int r = 0; r < R; ++r) {
+      long long take = s_ge[r] - s_gt[r];
       if (take > rem) take = rem;
       if (take < 0) take = 0;
       rem -= take;
-      const long long n = s_gt[l] + take;
-      n_keep[(long long)b * L + l] = (int32_t)n;
-      offsets[(long long)b * (L + 1) + l] = off;
+      const long long n = floor + s_gt[r] + take;
+      n_keep[(long long)b * R + r] = (int32_t)n;
+      offsets[(long long)b * (R + 1) + r] = off;
       off += n;
     }
-    offsets[(long long)b * (L + 1) + L] = off;
+    offsets[(long long)b * (R + 1) + R] = off;
   }
 }
 
@@ -191,30 +207,44 @@ size_t allocate_workspace_bytes(const Problem& P) {
   return align_up((size_t)P.Bt * 4 * kRadix * sizeof(unsigned int));
 }
 
-kvc_status launch_allocate(const Problem& P, const float* composite, long long budget,
-                           int32_t* n_keep, long long* offsets, void* ws, size_t ws_bytes,
-                           cudaStream_t st) {
+kvc_status launch_allocate(const Problem& P, const float* composite, long long budget, int heads_per_row,
+                           long long min_keep, int32_t* n_keep, long long* offsets, void* ws,
+                           size_t ws_bytes, cudaStream_t st) {
   if (ws_bytes < allocate_workspace_bytes(P)) {
     set_error("allocate: workspace too small");
     return KVC_ERR_WORKSPACE;
   }
+  const int R = P.L * heads_per_row;
+  if (R > kMaxSelectRows) {
+    set_error("allocate: %d rows in the pool, at most %d supported", R, kMaxSelectRows);
+    return KVC_ERR_UNSUPPORTED;
+  }
+  if (min_keep < 0 || min_keep > P.N || (long long)R * min_keep > budget) {
+    set_error("allocate: per-layer minimum %lld does not fit (N = %lld, rows * minimum <= budget = %lld required)",
+              min_keep, P.N, budget);
+    return KVC_ERR_INVALID_ARG;
+  }
+  const long long rest = budget - (long long)R * min_keep;     // handed out beyond the minimum
   unsigned int* hist = reinterpret_cast<unsigned int*>(ws);
   KVC_CUDA(launch_dependent(select_clear_kernel, dim3(P.Bt), dim3(4 * kRadix), 0, st, hist));
   KVC_LAUNCH_CHECK("select_clear_kernel");
-  const long long total = (long long)P.L * P.N;
+  const long long total = (long long)R * (P.N - min_keep);
   const long long tile = (long long)kHistThreads * kItemsPerThread;
   long long blocks = (total + tile - 1) / tile;
-  if (blocks > 592) blocks = 592;
+  int dev = 0, sms = 0;
+  KVC_CUDA(cudaGetDevice(&dev));
+  KVC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (blocks > 4LL * sms) blocks = 4LL * sms;
   if (blocks < 1) blocks = 1;
-  if (budget > 0) {
+  if (rest > 0) {
     for (int pass = 0; pass < 4; ++pass) {
       KVC_CUDA(launch_dependent(select_hist_kernel, dim3((unsigned)blocks, P.Bt), dim3(kHistThreads), 0, st,
-                                composite, hist, pass, P.L, P.Bt, P.N, budget));
+                                composite, hist, pass, R, P.Bt, heads_per_row, P.N, min_keep, rest));
       KVC_LAUNCH_CHECK("select_hist_kernel");
     }
   }
-  KVC_CUDA(launch_dependent(select_finish_kernel, dim3(P.Bt), dim3(1024), 0, st,
-                            composite, hist, P.L, P.Bt, P.N, budget, n_keep, offsets));
+  KVC_CUDA(launch_dependent(select_finish_kernel, dim3(P.Bt), dim3(1024), (size_t)R * 2 * sizeof(long long), st,
+                            composite, hist, R, P.Bt, heads_per_row, P.N, min_keep, rest, n_keep, offsets));
   KVC_LAUNCH_CHECK("select_finish_kernel");
   return KVC_OK;
 }

@@ -21,7 +21,7 @@ struct GatherParams {
   long long kvs0, kvs1, kvs2;  // in units of 16 bytes
   int lanes_per_row;           // row_bytes / 16
   int lanes_shift;             // log2(lanes_per_row)
-  long long rows_per_seq;      // budget * Hkv
+  long long rows_per_seq;      // budget * Hkv (per layer) or the budget in entries (per head)
 };
 
 __device__ inline uint4 ld_stream(const uint4* p) {
@@ -35,14 +35,18 @@ __device__ inline void st_stream(uint4* p, uint4 v) {
                :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// kPerHead = false: n_keep / offsets per layer, a layer's block is [Hkv, N_l, d] (Eqs. 23-24).
+// kPerHead = true:  n_keep / offsets per (layer, head), a head's block is [n, d] (App. A.2).
+template <bool kPerHead>
 __global__ void __launch_bounds__(kGatherThreads)
 gather_kernel(GatherParams P, LayerPtrs kp, LayerPtrs vp, const int32_t* __restrict__ idx,
               const int32_t* __restrict__ n_keep, const long long* __restrict__ offsets,
               uint4* __restrict__ k_out, uint4* __restrict__ v_out) {
-  __shared__ long long s_off[KVC_MAX_LAYERS + 1];
+  extern __shared__ long long s_off[];              // the sequence's offsets: R + 1 entries
   grid_dependency_wait();
   const int b = blockIdx.y;
-  for (int i = threadIdx.x; i <= P.L; i += kGatherThreads) s_off[i] = offsets[(long long)b * (P.L + 1) + i];
+  const int R = kPerHead ? P.L * P.Hkv : P.L;
+  for (int i = threadIdx.x; i <= R; i += kGatherThreads) s_off[i] = offsets[(long long)b * (R + 1) + i];
   __syncthreads();
 
   const int lpr = P.lanes_per_row;
@@ -58,17 +62,25 @@ gather_kernel(GatherParams P, LayerPtrs kp, LayerPtrs vp, const int32_t* __restr
       const long long r = row + u * rows_per_step;
       dst[u] = -1;
       if (r < P.rows_per_seq) {
-        // layer: the last l with offsets[l] * Hkv <= r
-        int lo = 0, hi = P.L;             // invariant: s_off[lo] * Hkv <= r < s_off[hi] * Hkv
+        // block: the last one whose first output row is <= r
+        const long long mult = kPerHead ? 1 : P.Hkv;
+        int lo = 0, hi = R;               // invariant: s_off[lo] * mult <= r < s_off[hi] * mult
         while (hi - lo > 1) {
           const int mid = (lo + hi) >> 1;
-          if (s_off[mid] * (long long)P.Hkv <= r) lo = mid; else hi = mid;
+          if (s_off[mid] * mult <= r) lo = mid; else hi = mid;
         }
-        const int l = lo;
-        const long long nl = n_keep[(long long)b * P.L + l];
-        const long long local = r - s_off[l] * P.Hkv;            // in [0, Hkv * nl)
-        const int h = (int)(local / nl);
-        const long long kk = local - (long long)h * nl;
+        int l, h;
+        long long kk;
+        if (kPerHead) {
+          l = lo / P.Hkv; h = lo - l * P.Hkv;
+          kk = r - s_off[lo];
+        } else {
+          l = lo;
+          const long long nl = n_keep[(long long)b * P.L + l];
+          const long long local = r - s_off[l] * P.Hkv;          // in [0, Hkv * nl)
+          h = (int)(local / nl);
+          kk = local - (long long)h * nl;
+        }
         const long long c = idx[(((long long)l * P.Bt + b) * P.Hkv + h) * P.N + kk];
         const long long src = b * P.kvs0 + h * P.kvs1 + c * P.kvs2 + sub;
         kv[u] = ld_stream(reinterpret_cast<const uint4*>(kp.p[l]) + src);
@@ -89,7 +101,7 @@ gather_kernel(GatherParams P, LayerPtrs kp, LayerPtrs vp, const int32_t* __restr
 }  // namespace
 
 kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& v, const int32_t* idx,
-                         const int32_t* n_keep, const long long* offsets, long long budget,
+                         const int32_t* n_keep, const long long* offsets, long long budget, bool per_head,
                          void* k_out, void* v_out, cudaStream_t st) {
   if (budget == 0) return KVC_OK;
   GatherParams gp;
@@ -100,15 +112,26 @@ kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& 
   gp.lanes_per_row = row_bytes / 16;
   gp.lanes_shift = 0;
   while ((1 << gp.lanes_shift) < gp.lanes_per_row) ++gp.lanes_shift;
-  gp.rows_per_seq = budget * P.Hkv;
+  gp.rows_per_seq = per_head ? budget : budget * P.Hkv;
   const long long rows_per_block = kGatherThreads / gp.lanes_per_row;
   long long blocks = (gp.rows_per_seq + rows_per_block * kUnroll - 1) / (rows_per_block * kUnroll);
-  const long long cap = 148LL * 128;   // measured best among 8 to 256 CTAs per SM's worth of grid
+  int dev = 0, sms = 0;
+  KVC_CUDA(cudaGetDevice(&dev));
+  KVC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const long long cap = (long long)sms * 128;   // measured best among 8 to 256 CTAs per SM's worth of grid
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  KVC_CUDA(launch_dependent(gather_kernel, dim3((unsigned)blocks, P.Bt), dim3(kGatherThreads), 0, st,
-                            gp, k, v, idx, n_keep, offsets, reinterpret_cast<uint4*>(k_out),
-                            reinterpret_cast<uint4*>(v_out)));
+  const int R = per_head ? P.L * P.Hkv : P.L;
+  const size_t smem = (size_t)(R + 1) * sizeof(long long);
+  if (per_head) {
+    KVC_CUDA(launch_dependent(gather_kernel<true>, dim3((unsigned)blocks, P.Bt), dim3(kGatherThreads), smem, st,
+                              gp, k, v, idx, n_keep, offsets, reinterpret_cast<uint4*>(k_out),
+                              reinterpret_cast<uint4*>(v_out)));
+  } else {
+    KVC_CUDA(launch_dependent(gather_kernel<false>, dim3((unsigned)blocks, P.Bt), dim3(kGatherThreads), smem, st,
+                              gp, k, v, idx, n_keep, offsets, reinterpret_cast<uint4*>(k_out),
+                              reinterpret_cast<uint4*>(v_out)));
+  }
   KVC_LAUNCH_CHECK("gather_kernel");
   return KVC_OK;
 }

@@ -36,18 +36,38 @@ static size_t score_scratch_bytes(const Problem& P) {
   return align_up(a);
 }
 
-size_t score_workspace_bytes(const Problem& P) { return score_scratch_bytes(P) + 256; }
+// [scratch][status word, 256 B][value norms, with the v-norm option]
+size_t score_workspace_bytes(const Problem& P) {
+  size_t n = score_scratch_bytes(P) + 256;
+  if (P.value_norm) n += align_up((size_t)P.L * P.Bt * P.Hkv * P.N * sizeof(float));
+  return n;
+}
 
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
-                        float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st) {
+                        float* scores, const float* vnorm, int* device_status, void* ws, size_t ws_bytes,
+                        cudaStream_t st) {
   if (score_sm100_supported(P)) {
     const float* parts = nullptr;
     int row_tiles = 1;
     const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st, &parts, &row_tiles);
-    if (s == KVC_OK) return launch_score_augment(P, scores, parts, row_tiles, st);
+    if (s == KVC_OK) return launch_score_augment(P, scores, parts, row_tiles, vnorm, st);
     if (s != KVC_ERR_UNSUPPORTED) return s;      // a real failure; UNSUPPORTED = strides TMA cannot take
   }
-  return launch_score_generic(P, gm, q, k, scores, ws, ws_bytes, st);
+  return launch_score_generic(P, gm, q, k, scores, vnorm, ws, ws_bytes, st);
+}
+
+// Scoring as the entry points run it: status word and value norms carved from the score workspace.
+static kvc_status run_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
+                            const LayerPtrs* v, float* scores, int* device_status, void* ws, cudaStream_t st) {
+  char* w = reinterpret_cast<char*>(ws);
+  const size_t scratch = score_scratch_bytes(P);
+  float* vnorm = nullptr;
+  if (P.value_norm) {
+    vnorm = reinterpret_cast<float*>(w + scratch + 256);
+    const kvc_status s = launch_value_norm(P, *v, vnorm, st);
+    if (s != KVC_OK) return s;
+  }
+  return launch_score(P, gm, q, k, scores, vnorm, device_status, ws, scratch, st);
 }
 
 namespace {
@@ -80,6 +100,12 @@ kvc_status resolve(const kvc_desc* d, Problem* P, GroupMap* gm) {
   KVC_REQUIRE(d->agg_group == KVC_AGG_MAX || d->agg_group == KVC_AGG_MEAN, KVC_ERR_INVALID_ARG, "bad agg_group");
   KVC_REQUIRE(d->agg_head == KVC_AGG_MAX || d->agg_head == KVC_AGG_MEAN, KVC_ERR_INVALID_ARG, "bad agg_head");
   KVC_REQUIRE(!(d->scale != d->scale) && !isinf(d->scale), KVC_ERR_INVALID_ARG, "scale is not finite");
+  KVC_REQUIRE(d->value_norm == 0 || d->value_norm == 1, KVC_ERR_INVALID_ARG, "value_norm must be 0 or 1");
+  KVC_REQUIRE(d->keep_position_order == 0 || d->keep_position_order == 1, KVC_ERR_INVALID_ARG,
+              "keep_position_order must be 0 or 1");
+  KVC_REQUIRE(d->min_keep_per_layer >= 0 && d->min_keep_per_layer <= d->n_ctx, KVC_ERR_INVALID_ARG,
+              "min_keep_per_layer must lie in [0, n_ctx]");
+  KVC_REQUIRE(d->reserved_ == 0, KVC_ERR_INVALID_ARG, "reserved_ must be 0");
 
   P->L = d->n_layers; P->Bt = d->batch; P->Hq = d->n_q_heads; P->Hkv = d->n_kv_heads;
   P->d = d->head_dim; P->w = d->window; P->N = d->n_ctx; P->q_pos0 = d->q_pos0;
@@ -87,6 +113,7 @@ kvc_status resolve(const kvc_desc* d, Problem* P, GroupMap* gm) {
   P->scale = (d->scale > 0.f) ? d->scale : 1.0f / sqrtf((float)d->head_dim);
   P->agg_task = d->agg_task; P->agg_group = d->agg_group; P->agg_head = d->agg_head;
   P->augment = d->augment_head_mean ? 1 : 0;
+  P->value_norm = d->value_norm; P->min_keep = d->min_keep_per_layer; P->keep_position_order = d->keep_position_order;
 
   if (d->q_stride[0] == 0) {
     P->qs[2] = P->d; P->qs[1] = (long long)P->w * P->d; P->qs[0] = P->qs[1] * P->Hq;
@@ -189,8 +216,12 @@ CompressLayout compress_layout(const Problem& P) {
   c.idx = off; off += align_up(items * 4);
   c.composite = off; off += align_up((size_t)P.L * P.Bt * P.N * 4);
   c.stage = off;
-  const size_t a = score_workspace_bytes(P), b = compose_workspace_bytes(P);
-  off += align_up(a > b ? a : b);
+  // (the bitmap of kvc_order_kept also lives here: the sort buffers are dead by then)
+  size_t a = score_workspace_bytes(P);
+  const size_t b = compose_workspace_bytes(P), o = order_kept_workspace_bytes(P);
+  if (b > a) a = b;
+  if (o > a) a = o;
+  off += align_up(a);
   c.alloc = off; off += align_up(allocate_workspace_bytes(P));
   c.total = off;
   return c;
@@ -254,12 +285,30 @@ kvc_status kvc_score(const kvc_desc* d, const void* const* q, const void* const*
   if ((s = check_ptrs(q, P.L, "q", &qp)) != KVC_OK) return s;
   if ((s = check_ptrs(k, P.L, "k", &kp)) != KVC_OK) return s;
   KVC_REQUIRE(scores != nullptr, KVC_ERR_INVALID_ARG, "scores is NULL");
+  KVC_REQUIRE(!P.value_norm, KVC_ERR_INVALID_ARG, "desc->value_norm is set: kvc_score has no V, use kvc_score_weighted");
   if ((s = check_ws(ws, ws_bytes, score_workspace_bytes(P))) != KVC_OK) return s;
   if ((s = check_device()) != KVC_OK) return s;
   // conditions detected on the device are reported in a word behind the scratch (kvc_score_status_offset)
   int* status = reinterpret_cast<int*>(reinterpret_cast<char*>(ws) + score_scratch_bytes(P));
   KVC_CUDA(cudaMemsetAsync(status, 0, sizeof(int), (cudaStream_t)stream));
-  return launch_score(P, gm, qp, kp, scores, status, ws, score_scratch_bytes(P), (cudaStream_t)stream);
+  return run_score(P, gm, qp, kp, nullptr, scores, status, ws, (cudaStream_t)stream);
+}
+
+kvc_status kvc_score_weighted(const kvc_desc* d, const void* const* q, const void* const* k,
+                              const void* const* v, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  Problem P; GroupMap gm; LayerPtrs qp, kp, vp;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  P.value_norm = 1;                               // (the descriptor's flag is ignored here)
+  if ((s = check_ptrs(q, P.L, "q", &qp)) != KVC_OK) return s;
+  if ((s = check_ptrs(k, P.L, "k", &kp)) != KVC_OK) return s;
+  if ((s = check_ptrs(v, P.L, "v", &vp)) != KVC_OK) return s;
+  KVC_REQUIRE(scores != nullptr, KVC_ERR_INVALID_ARG, "scores is NULL");
+  if ((s = check_ws(ws, ws_bytes, score_workspace_bytes(P))) != KVC_OK) return s;
+  if ((s = check_device()) != KVC_OK) return s;
+  int* status = reinterpret_cast<int*>(reinterpret_cast<char*>(ws) + score_scratch_bytes(P));
+  KVC_CUDA(cudaMemsetAsync(status, 0, sizeof(int), (cudaStream_t)stream));
+  return run_score(P, gm, qp, kp, &vp, scores, status, ws, (cudaStream_t)stream);
 }
 
 kvc_status kvc_score_status_offset(const kvc_desc* d, size_t* offset) {
@@ -291,8 +340,19 @@ kvc_status kvc_allocate(const kvc_desc* d, const float* composite, int64_t budge
   if ((s = check_budget(P, budget)) != KVC_OK) return s;
   if ((s = check_ws(ws, ws_bytes, allocate_workspace_bytes(P))) != KVC_OK) return s;
   if ((s = check_device()) != KVC_OK) return s;
-  return launch_allocate(P, composite, budget, n_keep, reinterpret_cast<long long*>(offsets), ws,
+  return launch_allocate(P, composite, budget, 1, P.min_keep, n_keep, reinterpret_cast<long long*>(offsets), ws,
                          ws_bytes, (cudaStream_t)stream);
+}
+
+kvc_status kvc_order_kept(const kvc_desc* d, int32_t* idx, const int32_t* n_keep, void* ws, size_t ws_bytes,
+                          void* stream) {
+  Problem P; GroupMap gm;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  KVC_REQUIRE(idx && n_keep, KVC_ERR_INVALID_ARG, "idx or n_keep is NULL");
+  if ((s = check_ws(ws, ws_bytes, order_kept_workspace_bytes(P))) != KVC_OK) return s;
+  if ((s = check_device()) != KVC_OK) return s;
+  return launch_order_kept(P, idx, n_keep, false, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 kvc_status kvc_gather(const kvc_desc* d, const void* const* k, const void* const* v, const int32_t* idx,
@@ -311,7 +371,7 @@ kvc_status kvc_gather(const kvc_desc* d, const void* const* k, const void* const
                 KVC_ERR_INVALID_ARG, "k_out / v_out must be 16-byte aligned");
   }
   if ((s = check_device()) != KVC_OK) return s;
-  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget,
+  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget, false,
                        k_out, v_out, (cudaStream_t)stream);
 }
 
@@ -345,11 +405,111 @@ kvc_status kvc_compress(const kvc_desc* d, const void* const* q, const void* con
   const size_t stage_bytes = lay.alloc - lay.stage;
 
   if (device_status) KVC_CUDA(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
-  if ((s = launch_score(P, gm, qp, kp, scores, device_status, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
+  if ((s = run_score(P, gm, qp, kp, &vp, scores, device_status, w + lay.stage, st)) != KVC_OK) return s;
   if ((s = launch_compose(P, scores, idx, composite, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
-  if ((s = launch_allocate(P, composite, budget, n_keep, reinterpret_cast<long long*>(offsets),
+  if ((s = launch_allocate(P, composite, budget, 1, P.min_keep, n_keep, reinterpret_cast<long long*>(offsets),
                            w + lay.alloc, lay.total - lay.alloc, st)) != KVC_OK) return s;
-  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget,
+  if (P.keep_position_order &&
+      (s = launch_order_kept(P, idx, n_keep, false, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
+  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget, false,
+                       k_out, v_out, st);
+}
+
+// ---- the unstructured variant (App. A.2) ----------------------------------------------------------
+
+static kvc_status check_entries(const Problem& P, long long budget_entries) {
+  KVC_REQUIRE(budget_entries >= 0 && budget_entries <= (long long)P.L * P.Hkv * P.N, KVC_ERR_INVALID_ARG,
+              "budget_entries %lld outside [0, L * Hkv * N = %lld]", budget_entries, (long long)P.L * P.Hkv * P.N);
+  KVC_REQUIRE(P.L * P.Hkv <= kMaxSelectRows, KVC_ERR_UNSUPPORTED, "L * Hkv = %d exceeds %d", P.L * P.Hkv,
+              kMaxSelectRows);
+  return KVC_OK;
+}
+
+// Ranking, the heads' sorted scores (into `sorted`), and the global selection over (layer, head).
+static kvc_status run_select_unstructured(const Problem& P, const float* scores, long long budget_entries,
+                                          int32_t* idx, int32_t* n_keep, long long* offsets, float* sorted,
+                                          char* w, const CompressLayout& lay, cudaStream_t st) {
+  kvc_status s;
+  const size_t stage_bytes = lay.alloc - lay.stage;
+  if ((s = launch_compose(P, scores, idx, nullptr, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
+  if ((s = launch_sorted_scores(P, w + lay.stage, sorted, st)) != KVC_OK) return s;
+  return launch_allocate(P, sorted, budget_entries, P.Hkv, 0, n_keep, offsets, w + lay.alloc, lay.total - lay.alloc, st);
+}
+
+kvc_status kvc_select_unstructured(const kvc_desc* d, const float* scores, int64_t budget_entries, int32_t* idx,
+                                   int32_t* n_keep, int64_t* offsets, void* ws, size_t ws_bytes, void* stream) {
+  Problem P; GroupMap gm;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  KVC_REQUIRE(scores && idx && n_keep && offsets, KVC_ERR_INVALID_ARG, "scores, idx, n_keep or offsets is NULL");
+  if ((s = check_entries(P, budget_entries)) != KVC_OK) return s;
+  const CompressLayout lay = compress_layout(P);
+  if ((s = check_ws(ws, ws_bytes, lay.total)) != KVC_OK) return s;
+  if ((s = check_device()) != KVC_OK) return s;
+  char* w = reinterpret_cast<char*>(ws);
+  // the caller's scores are not in the workspace, so its score region is free for the sorted scores
+  return run_select_unstructured(P, scores, budget_entries, idx, n_keep, reinterpret_cast<long long*>(offsets),
+                                 reinterpret_cast<float*>(w + lay.scores), w, lay, (cudaStream_t)stream);
+}
+
+kvc_status kvc_gather_unstructured(const kvc_desc* d, const void* const* k, const void* const* v,
+                                   const int32_t* idx, const int32_t* n_keep, const int64_t* offsets,
+                                   int64_t budget_entries, void* k_out, void* v_out, void* stream) {
+  Problem P; GroupMap gm; LayerPtrs kp, vp;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  if ((s = check_ptrs(k, P.L, "k", &kp)) != KVC_OK) return s;
+  if ((s = check_ptrs(v, P.L, "v", &vp)) != KVC_OK) return s;
+  KVC_REQUIRE(idx && n_keep && offsets, KVC_ERR_INVALID_ARG, "idx, n_keep or offsets is NULL");
+  if ((s = check_entries(P, budget_entries)) != KVC_OK) return s;
+  if (budget_entries > 0) {
+    KVC_REQUIRE(k_out && v_out, KVC_ERR_INVALID_ARG, "k_out or v_out is NULL");
+    KVC_REQUIRE(((reinterpret_cast<uintptr_t>(k_out) | reinterpret_cast<uintptr_t>(v_out)) & 15u) == 0,
+                KVC_ERR_INVALID_ARG, "k_out / v_out must be 16-byte aligned");
+  }
+  if ((s = check_device()) != KVC_OK) return s;
+  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget_entries, true,
+                       k_out, v_out, (cudaStream_t)stream);
+}
+
+kvc_status kvc_compress_unstructured(const kvc_desc* d, const void* const* q, const void* const* k,
+                                     const void* const* v, int64_t budget_entries, void* k_out, void* v_out,
+                                     int32_t* n_keep, int64_t* offsets, int32_t* idx_out, float* scores_out,
+                                     int32_t* device_status, void* ws, size_t ws_bytes, void* stream) {
+  Problem P; GroupMap gm; LayerPtrs qp, kp, vp;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  if ((s = check_ptrs(q, P.L, "q", &qp)) != KVC_OK) return s;
+  if ((s = check_ptrs(k, P.L, "k", &kp)) != KVC_OK) return s;
+  if ((s = check_ptrs(v, P.L, "v", &vp)) != KVC_OK) return s;
+  KVC_REQUIRE(n_keep && offsets, KVC_ERR_INVALID_ARG, "n_keep or offsets is NULL");
+  if ((s = check_entries(P, budget_entries)) != KVC_OK) return s;
+  if (budget_entries > 0) {
+    KVC_REQUIRE(k_out && v_out, KVC_ERR_INVALID_ARG, "k_out or v_out is NULL");
+    KVC_REQUIRE(((reinterpret_cast<uintptr_t>(k_out) | reinterpret_cast<uintptr_t>(v_out)) & 15u) == 0,
+                KVC_ERR_INVALID_ARG, "k_out / v_out must be 16-byte aligned");
+  }
+  const CompressLayout lay = compress_layout(P);
+  if ((s = check_ws(ws, ws_bytes, lay.total)) != KVC_OK) return s;
+  if ((s = check_device()) != KVC_OK) return s;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w = reinterpret_cast<char*>(ws);
+  float* scores = scores_out ? scores_out : reinterpret_cast<float*>(w + lay.scores);
+  int32_t* idx = idx_out ? idx_out : reinterpret_cast<int32_t*>(w + lay.idx);
+  // the sorted scores: the workspace's score region if the scores themselves go to the caller,
+  // else the composite-score region and what follows it cannot hold them -- they take the place of
+  // the scores, which nobody reads after the ranking
+  float* sorted = reinterpret_cast<float*>(w + lay.scores);
+  const size_t stage_bytes = lay.alloc - lay.stage;
+
+  if (device_status) KVC_CUDA(cudaMemsetAsync(device_status, 0, sizeof(int32_t), st));
+  if ((s = run_score(P, gm, qp, kp, &vp, scores, device_status, w + lay.stage, st)) != KVC_OK) return s;
+  if ((s = run_select_unstructured(P, scores, budget_entries, idx, n_keep, reinterpret_cast<long long*>(offsets),
+                                   sorted, w, lay, st)) != KVC_OK) return s;
+  if (P.keep_position_order &&
+      (s = launch_order_kept(P, idx, n_keep, true, w + lay.stage, stage_bytes, st)) != KVC_OK) return s;
+  return launch_gather(P, kp, vp, idx, n_keep, reinterpret_cast<const long long*>(offsets), budget_entries, true,
                        k_out, v_out, st);
 }
 

@@ -23,7 +23,10 @@ struct Problem {
   int elem_bytes;                 // 2 or 4
   int max_group;                  // largest number of query heads sharing one KV head
   bool contiguous_groups;         // q_to_kv[j] == j / G
+  int value_norm, min_keep, keep_position_order;   // the options of kvc_desc
 };
+
+constexpr int kMaxSelectRows = 2048;   // rows (layers, or layer-head pairs) of one sequence's selection pool
 
 // Query heads grouped by KV head: members of KV head h are qh[begin[h] .. begin[h+1]).
 struct GroupMap {
@@ -90,18 +93,21 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 // Scratch bytes the scoring step needs.
 size_t score_workspace_bytes(const Problem& P);
 // Eqs. 3, 14-16: writes scores [L, Bt, Hkv, N].
+// vnorm: nullptr, or ||v|| per (layer, sequence, KV head, token), laid out like scores (App. A.1.3).
 kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q, const LayerPtrs& k,
-                        float* scores, int* device_status, void* ws, size_t ws_bytes, cudaStream_t st);
+                        float* scores, const float* vnorm, int* device_status, void* ws, size_t ws_bytes,
+                        cudaStream_t st);
 // The two implementations behind it: CUDA cores (any supported shape) and tcgen05 (bf16,
 // contiguous GQA groups, window of at most 128 rows).
 size_t score_generic_workspace_bytes(const Problem& P);
 kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
-                                const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,
-                                cudaStream_t st);
+                                const LayerPtrs& k, float* scores, const float* vnorm, void* ws,
+                                size_t ws_bytes, cudaStream_t st);
 // Eq. 16 in place; before it, with `row_tiles` > 1, the group aggregate (Eq. 15) of every KV head
 // from its row tiles' partial aggregates `parts` [row_tiles][L*Bt*Hkv][N], in tile order.
+// With vnorm, the group aggregate is multiplied by the token's value norm before Eq. 16.
 kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
-                                cudaStream_t st);
+                                const float* vnorm, cudaStream_t st);
 bool score_sm100_supported(const Problem& P);
 size_t score_sm100_workspace_bytes(const Problem& P);
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
@@ -114,18 +120,35 @@ size_t compose_workspace_bytes(const Problem& P);
 kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, float* composite,
                           void* ws, size_t ws_bytes, cudaStream_t st);
 
+// Eq. 18 as fp32: the sorted scores of every head, from the keys the ranking leaves in the workspace
+// of launch_compose (which must have run on the same workspace).
+kvc_status launch_sorted_scores(const Problem& P, const void* ws, float* sorted, cudaStream_t st);
+
 // ---- allocate ---------------------------------------------------------------------------------
 size_t allocate_workspace_bytes(const Problem& P);
-// Eqs. 20-22: n_keep [Bt, L], offsets [Bt, L + 1].
-kvc_status launch_allocate(const Problem& P, const float* composite, long long budget,
-                           int32_t* n_keep, long long* offsets, void* ws, size_t ws_bytes,
-                           cudaStream_t st);
+// Eqs. 20-22: n_keep [Bt, L], offsets [Bt, L + 1], with the per-layer minimum `min_keep`.
+// heads_per_row = 1: the pool's rows are the layers, composite [L, Bt, N].  heads_per_row = Hkv (the
+// unstructured variant, App. A.2): the rows are the (layer, head) pairs, composite = the heads'
+// sorted scores [L, Bt, Hkv, N], n_keep [Bt, L * Hkv], offsets [Bt, L * Hkv + 1].
+kvc_status launch_allocate(const Problem& P, const float* composite, long long budget, int heads_per_row,
+                           long long min_keep, int32_t* n_keep, long long* offsets, void* ws,
+                           size_t ws_bytes, cudaStream_t st);
 
 // ---- gather -----------------------------------------------------------------------------------
 // Eqs. 23-24.
+// per_head: n_keep / offsets are per (layer, head) and `budget` counts entries (App. A.2).
 kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& v, const int32_t* idx,
-                         const int32_t* n_keep, const long long* offsets, long long budget,
+                         const int32_t* n_keep, const long long* offsets, long long budget, bool per_head,
                          void* k_out, void* v_out, cudaStream_t st);
+
+// ---- variants ---------------------------------------------------------------------------------
+// ||v||_2 of every value row in fp32: vnorm [L, Bt, Hkv, N] (App. A.1.3).
+kvc_status launch_value_norm(const Problem& P, const LayerPtrs& v, float* vnorm, cudaStream_t st);
+// The first n_keep entries of every idx row in ascending position, in place.  n_keep per layer
+// [Bt, L] or, per_head, per (layer, head) [Bt, L * Hkv].
+size_t order_kept_workspace_bytes(const Problem& P);
+kvc_status launch_order_kept(const Problem& P, int32_t* idx, const int32_t* n_keep, bool per_head,
+                             void* ws, size_t ws_bytes, cudaStream_t st);
 
 // Order-preserving map from an fp32 score to an unsigned key whose ASCENDING order is the
 // score's DESCENDING order; -0 is folded onto +0 so that equal scores get equal keys.

@@ -240,6 +240,13 @@ __global__ void compose_kernel(const uint32_t* __restrict__ keys, float* __restr
   composite[i] = acc;
 }
 
+// Eq. 18 as fp32: the sorted keys turned back into scores.
+__global__ void sorted_scores_kernel(const uint32_t* __restrict__ keys, float* __restrict__ sorted, long long total) {
+  grid_dependency_wait();
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) sorted[i] = key_to_score(keys[i]);
+}
+
 }  // namespace
 
 static int sort_tiles(const Problem& P) { return (int)((P.N + kTileItems - 1) / kTileItems); }
@@ -248,6 +255,15 @@ size_t compose_workspace_bytes(const Problem& P) {
   const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
   const size_t segments = (size_t)P.L * P.Bt * P.Hkv;
   return 4 * align_up(items * 4) + align_up(segments * sort_tiles(P) * kRadix * sizeof(uint32_t));
+}
+
+kvc_status launch_sorted_scores(const Problem& P, const void* ws, float* sorted, cudaStream_t st) {
+  const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
+  const uint32_t* keys_b = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(ws) + 2 * align_up(items * 4));
+  KVC_CUDA(launch_dependent(sorted_scores_kernel, dim3((unsigned)((items + 255) / 256)), dim3(256), 0, st,
+                            keys_b, sorted, (long long)items));
+  KVC_LAUNCH_CHECK("sorted_scores_kernel");
+  return KVC_OK;
 }
 
 kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, float* composite,
@@ -280,6 +296,7 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
                               scores, buf, idx, counts, P.N, tiles, pass));
     KVC_LAUNCH_CHECK("sort_scatter_kernel");
   }
+  if (composite == nullptr) return KVC_OK;      // ranking only (the unstructured variant has no Eq. 19)
   const long long total = (long long)P.L * P.Bt * P.N;
   KVC_CUDA(launch_dependent(compose_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
                             buf.keys_b, composite, P.Hkv, P.N, total, P.agg_head));

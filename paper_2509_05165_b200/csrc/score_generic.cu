@@ -241,23 +241,31 @@ score_emit_kernel(ScoreParams P, GroupMap gm, LayerPtrs qp, LayerPtrs kp,
 
 // Eq. 16: S[h, c] = S_group[h, c] + (1/Hkv) sum_i S_group[i, c], in place.  With row tiles, first
 // Eq. 15 from the tiles' partial aggregates (sum or max over the tile's query heads), in tile order.
+// With vnorm (App. A.1.3), the group aggregate is multiplied by the token's value norm before Eq. 16.
 __global__ void score_augment_kernel(float* __restrict__ s, const float* __restrict__ parts, int row_tiles,
-                                     int G, int agg_group, int augment, int Hkv, long long N, long long total) {
+                                     const float* __restrict__ vnorm, int G, int agg_group, int augment, int Hkv,
+                                     long long N, long long total) {
   grid_dependency_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const long long lb = i / N, c = i - lb * N;
   float* base = s + lb * Hkv * N + c;
-  if (row_tiles > 1) {
+  if (row_tiles > 1 || vnorm != nullptr) {
     const long long tile_stride = (total / N) * Hkv * N;          // one [L*Bt*Hkv][N] block per row tile
     const float* pbase = parts + lb * Hkv * N + c;
     for (int h = 0; h < Hkv; ++h) {
-      float acc = pbase[(long long)h * N];
-      for (int t = 1; t < row_tiles; ++t) {
-        const float v = pbase[(long long)t * tile_stride + (long long)h * N];
-        acc = (agg_group == KVC_AGG_MAX) ? fmaxf(acc, v) : acc + v;
+      float acc;
+      if (row_tiles > 1) {
+        acc = pbase[(long long)h * N];
+        for (int t = 1; t < row_tiles; ++t) {
+          const float v = pbase[(long long)t * tile_stride + (long long)h * N];
+          acc = (agg_group == KVC_AGG_MAX) ? fmaxf(acc, v) : acc + v;
+        }
+        if (agg_group == KVC_AGG_MEAN) acc = acc / (float)G;
+      } else {
+        acc = base[(long long)h * N];
       }
-      if (agg_group == KVC_AGG_MEAN) acc = acc / (float)G;
+      if (vnorm != nullptr) acc *= vnorm[lb * Hkv * N + (long long)h * N + c];
       base[(long long)h * N] = acc;
     }
   }
@@ -307,18 +315,18 @@ size_t score_generic_workspace_bytes(const Problem& P) {
 }
 
 kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
-                                cudaStream_t st) {
-  if (!P.augment && row_tiles <= 1) return KVC_OK;
+                                const float* vnorm, cudaStream_t st) {
+  if (!P.augment && row_tiles <= 1 && vnorm == nullptr) return KVC_OK;
   const long long total = (long long)P.L * P.Bt * P.N;
   KVC_CUDA(launch_dependent(score_augment_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                            scores, parts, row_tiles, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total));
+                            scores, parts, row_tiles, vnorm, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total));
   KVC_LAUNCH_CHECK("score_augment_kernel");
   return KVC_OK;
 }
 
 kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const LayerPtrs& q,
-                                const LayerPtrs& k, float* scores, void* ws, size_t ws_bytes,
-                                cudaStream_t st) {
+                                const LayerPtrs& k, float* scores, const float* vnorm, void* ws,
+                                size_t ws_bytes, cudaStream_t st) {
   if (ws_bytes < score_generic_workspace_bytes(P)) {
     set_error("score: workspace too small");
     return KVC_ERR_WORKSPACE;
@@ -337,7 +345,7 @@ kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const Laye
     else s = run<float, 128>(P, gm, q, k, scores, partial, lse2, nchunks, st);
   }
   if (s != KVC_OK) return s;
-  return launch_score_augment(P, scores, nullptr, 1, st);
+  return launch_score_augment(P, scores, nullptr, 1, vnorm, st);
 }
 
 }  // namespace kvc
