@@ -141,6 +141,13 @@ KVC_API kvc_status kvc_score(const kvc_desc* desc, const void* const* q, const v
  * writes (host call; depends on the problem only). */
 KVC_API kvc_status kvc_score_status_offset(const kvc_desc* desc, size_t* offset);
 
+/* 1 if kvc_score / kvc_compress score this problem with the tensor-core kernel (bf16, contiguous GQA
+ * groups q_to_kv[j] = j / G, at most 112 layers), 0 if they take the CUDA-core kernels (fp32, explicit
+ * group maps, anything else) -- same results, an order of magnitude slower --, negative on a bad
+ * descriptor.  Host call.  Strides that a tensor map cannot express (found when the maps are encoded)
+ * also send a call to the CUDA-core kernels. */
+KVC_API int32_t kvc_score_uses_tensor_cores(const kvc_desc* desc);
+
 /*
  * kvc_score with value-norm weighting (App. A.1.3 "Effect of Value Norms on Token Scores", the
  * v-norm variant): A^(w)[m, c] = A[m, c] * ||v[kv(j), c]||_2 takes the place of A in Eqs. 14-16.

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     kvc_debug_score_hooks,
     kvc_score,
     kvc_score_status_offset,
+    kvc_score_uses_tensor_cores,
     kvc_score_weighted,
     kvc_select_unstructured,
     kvc_version,

@@ -72,6 +72,8 @@ def _load():
     lib.kvc_score_status_offset.restype = C.c_int
     lib.kvc_debug_score_hooks.argtypes = [i64, i32]
     lib.kvc_debug_score_hooks.restype = None
+    lib.kvc_score_uses_tensor_cores.argtypes = [dp]
+    lib.kvc_score_uses_tensor_cores.restype = i32
     lib.kvc_score_weighted.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
     lib.kvc_score_weighted.restype = C.c_int
     lib.kvc_order_kept.argtypes = [dp, vp, vp, vp, sz, vp]
@@ -158,6 +160,14 @@ def kvc_score_weighted(desc, q, k, v, scores: torch.Tensor, workspace: torch.Ten
     wp, wb = _ws(workspace)
     _check(_load().kvc_score_weighted(C.byref(desc), _ptr_array(q), _ptr_array(k), _ptr_array(v), _dptr(scores),
                                       wp, wb, _stream(stream)))
+
+
+def kvc_score_uses_tensor_cores(desc: KvcDesc) -> bool:
+    """Whether scoring this problem runs on the tensor-core kernel (else on the CUDA-core kernels)."""
+    r = int(_load().kvc_score_uses_tensor_cores(C.byref(desc)))
+    if r < 0:
+        _check(r)
+    return r == 1
 
 
 def kvc_score_status_offset(desc: KvcDesc) -> int:

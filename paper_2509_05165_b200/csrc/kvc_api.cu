@@ -29,7 +29,7 @@ void count_launch(int n) { g_launches += n; }
 // Scratch of the scoring kernels; kvc_score keeps its device status word right behind it.
 static size_t score_scratch_bytes(const Problem& P) {
   size_t a = score_generic_workspace_bytes(P);
-  if (score_sm100_supported(P)) {
+  if (score_sm100_shape_ok(P)) {          // (by the shape alone: the size must not depend on the machine)
     const size_t b = score_sm100_workspace_bytes(P);
     if (b > a) a = b;
   }
@@ -48,9 +48,10 @@ kvc_status launch_score(const Problem& P, const GroupMap& gm, const LayerPtrs& q
                         cudaStream_t st) {
   if (score_sm100_supported(P)) {
     const float* parts = nullptr;
-    int row_tiles = 1;
-    const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st, &parts, &row_tiles);
-    if (s == KVC_OK) return launch_score_augment(P, scores, parts, row_tiles, vnorm, st);
+    int row_tiles = 1, tiles_per_head = 1;
+    const kvc_status s = launch_score_sm100(P, q, k, scores, device_status, ws, ws_bytes, st, &parts, &row_tiles,
+                                            &tiles_per_head);
+    if (s == KVC_OK) return launch_score_augment(P, scores, parts, row_tiles, tiles_per_head, vnorm, st);
     if (s != KVC_ERR_UNSUPPORTED) return s;      // a real failure; UNSUPPORTED = strides TMA cannot take
   }
   return launch_score_generic(P, gm, q, k, scores, vnorm, ws, ws_bytes, st);
@@ -309,6 +310,13 @@ kvc_status kvc_score_weighted(const kvc_desc* d, const void* const* q, const voi
   int* status = reinterpret_cast<int*>(reinterpret_cast<char*>(ws) + score_scratch_bytes(P));
   KVC_CUDA(cudaMemsetAsync(status, 0, sizeof(int), (cudaStream_t)stream));
   return run_score(P, gm, qp, kp, &vp, scores, status, ws, (cudaStream_t)stream);
+}
+
+int32_t kvc_score_uses_tensor_cores(const kvc_desc* d) {
+  Problem P; GroupMap gm;
+  const kvc_status s = resolve(d, &P, &gm);
+  if (s != KVC_OK) return (int32_t)s;
+  return score_sm100_shape_ok(P) ? 1 : 0;
 }
 
 kvc_status kvc_score_status_offset(const kvc_desc* d, size_t* offset) {

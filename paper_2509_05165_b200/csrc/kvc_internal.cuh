@@ -105,14 +105,17 @@ kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const Laye
                                 size_t ws_bytes, cudaStream_t st);
 // Eq. 16 in place; before it, with `row_tiles` > 1, the group aggregate (Eq. 15) of every KV head
 // from its row tiles' partial aggregates `parts` [row_tiles][L*Bt*Hkv][N], in tile order.
-// With vnorm, the group aggregate is multiplied by the token's value norm before Eq. 16.
+// With vnorm, the group aggregate is multiplied by the token's value norm before Eq. 16.  With
+// tiles_per_head > 1 (windows longer than 128 rows) every row tile holds a query head's partial
+// Eq. 14, and Eq. 14 is completed over a head's tiles before Eq. 15.
 kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
-                                const float* vnorm, cudaStream_t st);
+                                int tiles_per_head, const float* vnorm, cudaStream_t st);
+bool score_sm100_shape_ok(const Problem& P);
 bool score_sm100_supported(const Problem& P);
 size_t score_sm100_workspace_bytes(const Problem& P);
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
                               int* device_status, void* ws, size_t ws_bytes, cudaStream_t st,
-                              const float** parts_out, int* row_tiles_out);
+                              const float** parts_out, int* row_tiles_out, int* tiles_per_head_out);
 
 // ---- rank + compose ---------------------------------------------------------------------------
 size_t compose_workspace_bytes(const Problem& P);

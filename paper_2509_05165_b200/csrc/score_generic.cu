@@ -242,9 +242,12 @@ score_emit_kernel(ScoreParams P, GroupMap gm, LayerPtrs qp, LayerPtrs kp,
 // Eq. 16: S[h, c] = S_group[h, c] + (1/Hkv) sum_i S_group[i, c], in place.  With row tiles, first
 // Eq. 15 from the tiles' partial aggregates (sum or max over the tile's query heads), in tile order.
 // With vnorm (App. A.1.3), the group aggregate is multiplied by the token's value norm before Eq. 16.
+// With tiles_per_head > 1 (windows longer than 128 rows) a row tile holds one query head's partial
+// Eq. 14 -- the maximum or the sum of the attention weights over the tile's rows -- and Eq. 14 is
+// completed over the head's tiles (the sum divided by w) before Eq. 15, heads in ascending order.
 __global__ void score_augment_kernel(float* __restrict__ s, const float* __restrict__ parts, int row_tiles,
-                                     const float* __restrict__ vnorm, int G, int agg_group, int augment, int Hkv,
-                                     long long N, long long total) {
+                                     int tiles_per_head, int agg_task, int w, const float* __restrict__ vnorm, int G,
+                                     int agg_group, int augment, int Hkv, long long N, long long total) {
   grid_dependency_wait();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
@@ -255,7 +258,19 @@ __global__ void score_augment_kernel(float* __restrict__ s, const float* __restr
     const float* pbase = parts + lb * Hkv * N + c;
     for (int h = 0; h < Hkv; ++h) {
       float acc;
-      if (row_tiles > 1) {
+      if (row_tiles > 1 && tiles_per_head > 1) {
+        acc = (agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
+        for (int j = 0; j < row_tiles / tiles_per_head; ++j) {       // the query heads of the group
+          float ht = pbase[(long long)(j * tiles_per_head) * tile_stride + (long long)h * N];
+          for (int t = 1; t < tiles_per_head; ++t) {
+            const float v = pbase[(long long)(j * tiles_per_head + t) * tile_stride + (long long)h * N];
+            ht = (agg_task == KVC_AGG_MAX) ? fmaxf(ht, v) : ht + v;
+          }
+          if (agg_task == KVC_AGG_MEAN) ht = ht / (float)w;
+          acc = (agg_group == KVC_AGG_MAX) ? fmaxf(acc, ht) : acc + ht;
+        }
+        if (agg_group == KVC_AGG_MEAN) acc = acc / (float)G;
+      } else if (row_tiles > 1) {
         acc = pbase[(long long)h * N];
         for (int t = 1; t < row_tiles; ++t) {
           const float v = pbase[(long long)t * tile_stride + (long long)h * N];
@@ -315,11 +330,12 @@ size_t score_generic_workspace_bytes(const Problem& P) {
 }
 
 kvc_status launch_score_augment(const Problem& P, float* scores, const float* parts, int row_tiles,
-                                const float* vnorm, cudaStream_t st) {
+                                int tiles_per_head, const float* vnorm, cudaStream_t st) {
   if (!P.augment && row_tiles <= 1 && vnorm == nullptr) return KVC_OK;
   const long long total = (long long)P.L * P.Bt * P.N;
   KVC_CUDA(launch_dependent(score_augment_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                            scores, parts, row_tiles, vnorm, P.max_group, P.agg_group, P.augment, P.Hkv, P.N, total));
+                            scores, parts, row_tiles, tiles_per_head, P.agg_task, P.w, vnorm, P.max_group, P.agg_group,
+                            P.augment, P.Hkv, P.N, total));
   KVC_LAUNCH_CHECK("score_augment_kernel");
   return KVC_OK;
 }
@@ -345,7 +361,7 @@ kvc_status launch_score_generic(const Problem& P, const GroupMap& gm, const Laye
     else s = run<float, 128>(P, gm, q, k, scores, partial, lse2, nchunks, st);
   }
   if (s != KVC_OK) return s;
-  return launch_score_augment(P, scores, nullptr, 1, vnorm, st);
+  return launch_score_augment(P, scores, nullptr, 1, 1, vnorm, st);
 }
 
 }  // namespace kvc

@@ -99,6 +99,8 @@ struct FastParams {
   float* scores;               // [L*Bt*Hkv][N], or with QT > 1 the partial aggregates [QT][L*Bt*Hkv][N]
   int L, Bt, Hkv, G;
   int HPT, QT, w;              // query heads per row tile, row tiles per KV head, window rows per query head
+  int CH;                      // row tiles per query head: 1, or ceil(w / 128) for windows longer than 128 rows
+                               // (then HPT = 1 and row tile q holds rows (q % CH) * 128 .. of query head q / CH)
   long long N, q_pos0;
   int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
   int RT;                      // tiles per run
@@ -346,7 +348,12 @@ struct Cursor {
     b = lb - l * P.Bt;
   }
   // window rows of this unit's row tile (whole query heads; the last tile of a KV head may be short)
-  __device__ __forceinline__ int rows(const FastParams& P) const { return min(P.HPT, P.G - q * P.HPT) * P.w; }
+  __device__ __forceinline__ int rows(const FastParams& P) const {
+    return P.CH == 1 ? min(P.HPT, P.G - q * P.HPT) * P.w : min(kRows, P.w - (q % P.CH) * kRows);
+  }
+  // first window row of this row tile inside its query head, and the tile's first query head in the group
+  __device__ __forceinline__ int row0(const FastParams& P) const { return P.CH == 1 ? 0 : (q % P.CH) * kRows; }
+  __device__ __forceinline__ int head0(const FastParams& P) const { return P.CH == 1 ? q * P.HPT : q / P.CH; }
   // index of the (layer, sequence, KV head)
   __device__ __forceinline__ int kv_unit(const FastParams& P) const { return (l * P.Bt + b) * P.Hkv + h; }
   __device__ __forceinline__ int tile(const FastParams& P) const { return j * P.RT + t; }
@@ -515,6 +522,29 @@ __device__ __noinline__ float p2_generic_tile(uint32_t taddr, const float* neg_l
   return gacc;
 }
 
+// Pass 2, one token against the R rows of one query head that this row tile holds (windows longer
+// than 128 rows), with masking: rows below m_min do not see the token.  Returns the tile's part of
+// Eq. 14 for the token: the largest attention weight, or the sum of the weights, over these rows.
+template <bool kTaskMean>
+__device__ __noinline__ float p2_long_tile(uint32_t taddr, const float* neg_lse, int n_chunks, int R, float sl2e,
+                                           bool full, long long m_min) {
+  float hacc = kTaskMean ? 0.f : -INFINITY;
+#pragma unroll 1
+  for (int j = 0; j < n_chunks; ++j) {
+    uint32_t r[32];
+    tc_ld32_nowait(taddr + j * 32, r);
+    tc_wait_ld(r);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int col = j * 32 + i;
+      float xi = fmaf(__uint_as_float(r[i]), sl2e, neg_lse[col]);       // log2 of the attention weight
+      if (col >= R || (!full && col < m_min)) xi = -INFINITY;
+      if (kTaskMean) hacc += ex2(xi); else hacc = fmaxf(hacc, xi);
+    }
+  }
+  return kTaskMean ? hacc : ex2(hacc);
+}
+
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
@@ -569,7 +599,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   }
   const int my_tiles = my_runs * P.RT;                  // stream length (some positions hold no tile)
   const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
-  const uint32_t q_bytes = (uint32_t)(P.HPT * P.w) * D * 2;   // the whole box arrives (rows outside the tensor as zeros)
+  // the whole box arrives (rows outside the tensor as zeros)
+  const uint32_t q_bytes = (uint32_t)(P.CH == 1 ? P.HPT * P.w : kRows) * D * 2;
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
   if (warp == 0) {
@@ -607,7 +638,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 mbar_expect_tx(bar_qfull(qr.i), q_bytes);
                 for (int hf = 0; hf < SL::kHalves; ++hf)
                   tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
-                              bar_qfull(qr.i), hf * 64, 0, c.h * P.G + c.q * P.HPT, c.b, pol_keep);
+                              bar_qfull(qr.i), hf * 64, c.row0(P), c.h * P.G + c.head0(P), c.b, pol_keep);
                 qr.next(kQSlots);
                 if (qc < kQSlots) ++qc;
               }
@@ -796,7 +827,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const int row = quarter * 32 + lane;              // TMEM lane = query row
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     float2* stage = reinterpret_cast<float2*>(smem + SL::kStats) + row;
-    const long long row_vis = min(P.N - 1, P.q_pos0 + (row % (W > 0 ? W : P.w)));     // last key this row sees
+    const int row_m = row % (W > 0 ? W : P.w);        // the row inside its query head (windows of up to 128 rows)
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
 
     int n1 = 0;
@@ -862,6 +893,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           if (row_used) { fast_chunk(ra); fast_chunk(rb); }
         } else {
           float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
+          const long long row_vis = min(P.N - 1, P.q_pos0 + (P.CH == 1 ? row_m : c.row0(P) + row));   // last key this row sees
           p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
           if (row_used) { mref = m2; lsum = l2; }
           tc_fence_before();
@@ -1021,6 +1053,14 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             hacc = -INFINITY;
           }
         }
+      } else if (W == 0 && P.CH > 1) {
+        // a window longer than 128 rows: the tile holds rows row0 .. of one query head and yields
+        // that head's partial Eq. 14 (the maximum, or the sum, over these rows)
+        gacc = p2_long_tile<kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
+                                       c - P.q_pos0 - cu.row0(P));
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(buf));
       } else {
         gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
                                              c - P.q_pos0, P.agg_group, P.w);
@@ -1051,7 +1091,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 // 2^(logit - ref) is then at least about 1, so fixed point with 20 fractional bits keeps it.
 // ------------------------------------------------------------------------------------------------
 struct RefParams {
-  int Bt, Hkv, G, HPT, QT, w, d, NG;
+  int Bt, Hkv, G, HPT, QT, CH, w, d, NG;
   unsigned long long* acc;     // [U][128]: cleared here
   int* group_counter;          // [U][NG], int* unit_counter [U], unsigned* lse2 [U][128]: preset here
   int* unit_counter;
@@ -1072,10 +1112,11 @@ score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ re
   const int uh = u / P.QT, qt = u - uh * P.QT;
   const int lb = uh / P.Hkv, h = uh - lb * P.Hkv;
   const int l = lb / P.Bt, b = lb - l * P.Bt;
-  const int rows_u = min(P.HPT, P.G - qt * P.HPT) * P.w;
+  const int rows_u = P.CH == 1 ? min(P.HPT, P.G - qt * P.HPT) * P.w : min(kRows, P.w - (qt % P.CH) * kRows);
   float r = 0.f;
   if (row < rows_u) {
-    const int j = h * P.G + qt * P.HPT + row / P.w, m = row % P.w;
+    const int j = P.CH == 1 ? h * P.G + qt * P.HPT + row / P.w : h * P.G + qt / P.CH;
+    const int m = P.CH == 1 ? row % P.w : (qt % P.CH) * kRows + row;
     const __nv_bfloat16* qv = reinterpret_cast<const __nv_bfloat16*>(qp.p[l]) + b * P.qs0 + j * P.qs1 + m * P.qs2;
     const __nv_bfloat16* kv = reinterpret_cast<const __nv_bfloat16*>(kp.p[l]) + b * P.kvs0 + h * P.kvs1;
     // 16-byte pieces (rows are 16-byte aligned), all in flight at once; products added in order
@@ -1132,7 +1173,7 @@ bool encode_map(CUtensorMap* m, const void* base, const long long dims[4], const
 
 struct FastPlan {
   int U, NT, RPU, NG, grid, RT;
-  int HPT, QT;                 // query heads per row tile, row tiles per KV head
+  int HPT, QT, CH;             // query heads per row tile, row tiles per KV head, row tiles per query head
   long long total_runs, shift;
   size_t off_partial, off_group, off_sync, sync_bytes, off_parts, off_acc, off_ref, off_total;
 };
@@ -1140,8 +1181,15 @@ struct FastPlan {
 // sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
 void make_plan(const Problem& P, int sms, FastPlan* pl) {
   const int G = P.Hq / P.Hkv;
-  pl->HPT = kRows / P.w < G ? kRows / P.w : G;
-  pl->QT = (G + pl->HPT - 1) / pl->HPT;
+  if (P.w <= kRows) {
+    pl->HPT = kRows / P.w < G ? kRows / P.w : G;
+    pl->CH = 1;
+    pl->QT = (G + pl->HPT - 1) / pl->HPT;
+  } else {                      // a window longer than one accumulator: several row tiles per query head
+    pl->HPT = 1;
+    pl->CH = (P.w + kRows - 1) / kRows;
+    pl->QT = G * pl->CH;
+  }
   pl->U = P.L * P.Bt * P.Hkv * pl->QT;
   pl->NT = (int)((P.N + kTile - 1) / kTile);
   pl->RT = kMinRunTiles;
@@ -1230,17 +1278,21 @@ kvc_status launch_w(int W, const FastParams& fp, int grid, cudaStream_t st) {
 
 }  // namespace
 
-bool score_sm100_supported(const Problem& P) {
+// The descriptor alone: is this a shape the tensor-core kernel handles?
+bool score_sm100_shape_ok(const Problem& P) {
   if (P.dtype != KVC_BF16 || !P.contiguous_groups) return false;
-  if (P.w < 1 || P.w > kRows) return false;
+  if (P.w < 1) return false;
   if (P.L > kMaxFastLayers) return false;
   if (P.N >= (1LL << 30)) return false;
   FastPlan pl;
   make_plan(P, 0, &pl);
   if ((long long)P.L * P.Bt * P.Hkv * pl.QT > (1 << 24)) return false;
   if ((pl.total_runs + 4096) * pl.RT + pl.shift >= (1LL << 31)) return false;   // 32-bit sequence indices
-  return encode_fn() != nullptr;
+  return true;
 }
+
+// ... and can its tensor maps be encoded here (a driver with the encoder is present)?
+bool score_sm100_supported(const Problem& P) { return score_sm100_shape_ok(P) && encode_fn() != nullptr; }
 
 size_t score_sm100_workspace_bytes(const Problem& P) {
   FastPlan pl;
@@ -1252,7 +1304,7 @@ size_t score_sm100_workspace_bytes(const Problem& P) {
 // for these strides; the caller then uses the CUDA-core path.
 kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerPtrs& k, float* scores,
                               int* device_status, void* ws, size_t ws_bytes, cudaStream_t st,
-                              const float** parts_out, int* row_tiles_out) {
+                              const float** parts_out, int* row_tiles_out, int* tiles_per_head_out) {
   const int sms = sm_count();
   if (sms < 1) return KVC_ERR_UNSUPPORTED;
   FastPlan pl;
@@ -1266,7 +1318,7 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
     const unsigned kb[4] = {64, (unsigned)kTile, 1, 1};
     const long long qd[4] = {P.d, P.w, P.Hq, P.Bt};
     const long long qs[3] = {P.qs[2] * 2, P.qs[1] * 2, P.qs[0] * 2};
-    const unsigned qb[4] = {64, (unsigned)P.w, (unsigned)pl.HPT, 1};
+    const unsigned qb[4] = {64, (unsigned)(pl.CH == 1 ? P.w : kRows), (unsigned)pl.HPT, 1};
     if (!encode_map(&fp.k_maps[l], k.p[l], kd, ks, kb)) return KVC_ERR_UNSUPPORTED;
     if (!encode_map(&fp.q_maps[l], q.p[l], qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
   }
@@ -1284,7 +1336,7 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
     RefParams rp;
     rp.NG = pl.NG; rp.acc = fp.acc; rp.group_counter = fp.group_counter; rp.unit_counter = fp.unit_counter;
     rp.lse2 = fp.lse2;
-    rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.w = P.w; rp.d = P.d;
+    rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.CH = pl.CH; rp.w = P.w; rp.d = P.d;
     rp.qs0 = P.qs[0]; rp.qs1 = P.qs[1]; rp.qs2 = P.qs[2]; rp.kvs0 = P.kvs[0]; rp.kvs1 = P.kvs[1];
     rp.sl2e = P.scale * kLog2eF;
     KVC_CUDA(launch_dependent(score_ref_kernel, dim3(pl.U), dim3(kRows), 0, st, rp, q, k, ref));
@@ -1295,8 +1347,9 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.scores = pl.QT > 1 ? parts : scores;
   *parts_out = parts;
   *row_tiles_out = pl.QT;
+  *tiles_per_head_out = pl.CH;
   fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G;
-  fp.HPT = pl.HPT; fp.QT = pl.QT; fp.w = P.w;
+  fp.HPT = pl.HPT; fp.QT = pl.QT; fp.CH = pl.CH; fp.w = P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
   fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.RT = pl.RT; fp.NG = pl.NG; fp.grid = pl.grid;
   fp.total_runs = (unsigned int)pl.total_runs; fp.shift = (int)pl.shift;

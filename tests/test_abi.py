@@ -61,6 +61,8 @@ def test_workspace_size_is_positive_and_monotone_in_n():
     ("n_layers", 0, -1), ("n_layers", 129, -2), ("batch", 0, -1), ("head_dim", 96, -2),
     ("window", 0, -1), ("n_ctx", 0, -1), ("n_ctx", 1 << 31, -2), ("q_pos0", -1, -1),
     ("dtype", 7, -1), ("agg_task", 2, -1), ("n_q_heads", 5, -1), ("n_kv_heads", 0, -1),
+    ("value_norm", 2, -1), ("keep_position_order", -1, -1), ("min_keep_per_layer", -1, -1),
+    ("min_keep_per_layer", 513, -1), ("reserved_", 1, -1),
 ])
 def test_bad_descriptors_are_rejected(field, value, status):
     d = kvc.kvc_desc_init(2, 1, 4, 2, 64, 512, 16, kvc.F32)
@@ -117,3 +119,20 @@ def test_no_cpu_fallback_without_a_gpu():
     with pytest.raises(kvc.KvcError) as e:
         kvc.kvc_score(d, q, k, S, ws[off:])
     assert e.value.status == -4
+
+
+def test_scoring_path_query_and_option_defaults():
+    d = kvc.kvc_desc_init(32, 1, 32, 8, 128, 32768, 32, kvc.BF16)
+    assert (d.value_norm, d.min_keep_per_layer, d.keep_position_order, d.reserved_) == (0, 0, 0, 0)
+    assert kvc.kvc_score_uses_tensor_cores(d)
+    assert kvc.kvc_score_uses_tensor_cores(kvc.kvc_desc_init(32, 1, 32, 8, 128, 32768, 1000, kvc.BF16))
+    assert not kvc.kvc_score_uses_tensor_cores(kvc.kvc_desc_init(2, 1, 4, 2, 64, 512, 16, kvc.F32))
+    m = (C.c_int32 * 4)(1, 0, 1, 0)
+    d2 = kvc.kvc_desc_init(2, 1, 4, 2, 64, 512, 16, kvc.BF16)
+    d2.q_to_kv = C.cast(m, C.POINTER(C.c_int32))
+    assert not kvc.kvc_score_uses_tensor_cores(d2)
+    # the v-norm option enlarges the workspace by the value norms
+    d3 = kvc.kvc_desc_init(2, 1, 4, 2, 64, 512, 16, kvc.BF16)
+    a = kvc.kvc_workspace_size(d3, 10)
+    d3.value_norm = 1
+    assert kvc.kvc_workspace_size(d3, 10) >= a

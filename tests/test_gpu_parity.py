@@ -223,6 +223,28 @@ def test_window_lengths_other_than_powers_of_two(Hq, Hkv, w, agg_task, agg_group
     check_all(wl, desc, cfg.budget)
 
 
+@pytest.mark.parametrize("Hq,Hkv,w,agg_task,agg_group,q_pos0", [
+    (4, 2, 200, 0, 1, 5000),     # task-aware: 200 task tokens after the context, two row tiles per query head
+    (4, 2, 300, 1, 0, 5000),     # three row tiles (the last one short), task mean, group max
+    (2, 1, 1000, 0, 1, 5000),    # a thousand task tokens: eight row tiles per query head
+    (4, 2, 300, 0, 1, None),     # the window is the end of the context: the causal mask runs through 300 rows
+    (6, 2, 130, 1, 1, 900),      # barely more than one tile; three query heads per KV head; mask inside
+])
+def test_windows_longer_than_one_accumulator_tile(Hq, Hkv, w, agg_task, agg_group, q_pos0):
+    """Hundreds to thousands of scoring rows per query head (the task-aware setting of Sec. 3.2.1):
+    a query head is cut into row tiles of 128 rows, Eq. 14 is completed over a head's tiles."""
+    dev = _cuda()
+    cfg = W.WorkloadConfig("longwin", 2, Hq, Hkv, 128, 1500, w, dtype="bf16", retention=0.3, elem_std=1.0,
+                           hh_frac=0.01)
+    wl = W.make_workload(cfg, dev)
+    kw = dict(agg_task=agg_task, agg_group=agg_group)
+    if q_pos0 is not None:
+        kw["q_pos0"] = q_pos0
+    desc = kvc.desc_from_config(cfg, **kw)
+    assert kvc.kvc_score_uses_tensor_cores(desc)
+    check_all(wl, desc, cfg.budget)
+
+
 @pytest.mark.parametrize("scale", [2.0, 0.5])
 def test_logits_far_above_the_first_tokens(scale):
     """A large logit scale: for most window rows some token lies tens of nats above token 0, whose
