@@ -9,6 +9,8 @@ LLaMA-3.1-8B-shaped cache at N = 32768, window 32, 25 % retention (the configura
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--retention R]
   python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...   (N > 1)
   python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
+  python bench.py --sweep                   # the N x batch x retention sweep on the 8B shape, one JSON line per point
+                                            # (points that do not fit the free device memory are recorded as skipped)
 
 Prints ONE JSON line on rank 0.  Multi-GPU: every rank compresses its own sequence (weak
 scaling, no data-path collective); the time is the max over ranks.
@@ -16,8 +18,10 @@ scaling, no data-path collective); the time is the max over ranks.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -51,6 +55,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU work of the oracle leg")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the second, long timed region (0 = leave it out)")
+    ap.add_argument("--sweep", action="store_true", help="run the N x batch x retention sweep instead of one workload")
     return ap.parse_args()
 
 
@@ -180,6 +187,32 @@ def time_oracle(cfg, q, k, kr, vr):
     return time.perf_counter() - t0
 
 
+def parity_summary(cfg, gpu_scores, gpu_idx):
+    """The GPU's scores and order of layer 0, sequence 0 against the all-double oracle (part of the
+    oracle leg, outside every timed region): largest relative score error, positions where the order
+    differs with the largest oracle score gap among them, and the smallest gap where both agree."""
+    import oracle
+
+    q, k, _, _ = oracle_sample(cfg, 1)
+    S_def = oracle.score_layer(q[0], k[0], 1.0 / np.sqrt(cfg.head_dim), cfg.n_ctx - cfg.window)
+    S_gpu = gpu_scores.astype(np.float64)
+    rel = np.abs(S_gpu - S_def) / np.maximum(np.abs(S_def), 1e-300)
+    n_diff, max_gap, margin = 0, 0.0, float("inf")
+    for h in range(S_def.shape[0]):
+        ref, Ss = oracle.rank(S_def[h])
+        diff = ref != gpu_idx[h]
+        n_diff += int(diff.sum())
+        if diff.any():
+            x, y = S_def[h][ref[diff]], S_def[h][gpu_idx[h][diff]]
+            max_gap = max(max_gap, float((np.abs(x - y) / np.maximum(x, y)).max()))
+        agree = ~diff[:-1] & ~diff[1:]
+        if agree.any():
+            margin = min(margin, float(((Ss[:-1] - Ss[1:])[agree] / Ss[:-1][agree]).min()))
+    return dict(layer=0, tolerance=1e-3, max_rel_score_err=float(rel[S_def > 0].max()), n_order_diff=n_diff,
+                max_gap_at_diff=max_gap, tie_margin=margin,
+                ok=bool(rel[S_def > 0].max() <= 1e-3 and max_gap < 2e-3))
+
+
 def cpu_baseline(cfg, target_seconds):
     """The oracle as it stands, on the host cores, on the first layers of the same workload."""
     import oracle
@@ -198,11 +231,14 @@ def cpu_baseline(cfg, target_seconds):
     return dict(value=cfg.n_ctx / per_pass, unit=UNIT, cores=cores, kind="oracle",
                 sample="%d of %d layers of %s, one sequence, whole pass incl. gather: %.2f s measured, "
                        "scaled linearly to all layers" % (Ls, cfg.n_layers, cfg.name, t),
-                seconds_measured=t)
+                seconds_measured=t, extrapolated=Ls < cfg.n_layers)
 
 
 def run_reference(args):
-    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only).  A step is the oracle's
+    whole pass over the first layers of the workload (two of them by default: the full workload would take
+    minutes per step); value and ms_per_step are scaled linearly to all layers and marked as extrapolated,
+    the measured time of a step is reported beside them."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import oracle
@@ -221,8 +257,10 @@ def run_reference(args):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=t_step * 1e3 * cfg.n_layers / Ls, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=workload_config(cfg, 1),
-                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                config=workload_config(cfg, 1), extrapolated=Ls < cfg.n_layers, layers_timed=Ls,
+                ms_per_step_measured=t_step * 1e3,
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample,
+                                  extrapolated=Ls < cfg.n_layers),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
@@ -246,11 +284,28 @@ def aggregate_tokens_per_s(cfg, world, ms_per_step):
     return cfg.batch * cfg.n_ctx * world / (ms_per_step * 1e-3)
 
 
-# DRAM traffic of one launch of the scoring kernel on the default workload, from the ncu capture
-# summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of a 4-layer capture,
-# scaled by 8 to the 32 layers of the workload: the traffic is proportional to the layers).
-# None for any other workload, and to be reset to None whenever the kernel changes.
-SCORE_TRAFFIC_BYTES = {"llama8b_32k": 8 * (273443072 + 8006912)}   # 2.25 GB: K leaves HBM once (1.04x algorithmic)
+SCORE_SOURCE = os.path.join(ROOT, "paper_2509_05165_b200", "csrc", "score_sm100.cu")
+SCORE_PROFILE = os.path.join(ROOT, "profiles", "score_sm100_llama8b_32k_L4.txt")
+
+
+def score_traffic_bytes(cfg):
+    """DRAM traffic of one launch of the scoring kernel on this workload, from the ncu capture summarised in
+    profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of a 4-layer capture of the same shape, scaled to
+    the workload's layers: the traffic is proportional to them).  None for any other shape, and None as soon
+    as the kernel's source is no longer the one the capture was taken on (the summary records its hash)."""
+    if not cfg.name.startswith("llama8b_32k") or cfg.n_ctx != 32768 or cfg.batch != 1:
+        return None
+    try:
+        text = open(SCORE_PROFILE).read()
+        sha = re.search(r"source_sha256:\s*([0-9a-f]{64})", text).group(1)
+        rd = int(re.search(r"dram_bytes_read_per_launch:\s*(\d+)", text).group(1))
+        wr = int(re.search(r"dram_bytes_write_per_launch:\s*(\d+)", text).group(1))
+        layers = int(re.search(r"capture_layers:\s*(\d+)", text).group(1))
+        if hashlib.sha256(open(SCORE_SOURCE, "rb").read()).hexdigest() != sha:
+            return None
+        return (rd + wr) * cfg.n_layers // layers
+    except Exception:  # noqa: BLE001
+        return None
 
 
 def workload_config(cfg, world):
@@ -263,28 +318,27 @@ def workload_config(cfg, world):
                     (2 if cfg.dtype == "bf16" else 4) / 1e9))
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
+def device_bytes_needed(cfg):
+    """Device memory one run of the benchmark holds for this workload: inputs, outputs, workspace, and the
+    kept intermediates of the per-stage timing."""
+    import paper_2509_05165_b200 as kvc
 
+    e = 2 if cfg.dtype == "bf16" else 4
+    kv = 2 * cfg.batch * cfg.n_layers * cfg.n_kv_heads * cfg.n_ctx * cfg.head_dim * e
+    q = cfg.batch * cfg.n_layers * cfg.n_q_heads * cfg.window * cfg.head_dim * e
+    outs = 2 * 2 * cfg.batch * cfg.budget * cfg.n_kv_heads * cfg.head_dim * e
+    inter = cfg.batch * cfg.n_layers * cfg.n_ctx * (8 * cfg.n_kv_heads + 4)
+    ws = kvc.kvc_workspace_size(kvc.desc_from_config(cfg), cfg.budget)
+    draw = cfg.batch * cfg.n_kv_heads * cfg.n_ctx * cfg.head_dim * 4 * 4      # fp32 temporaries of the generator
+    return kv + q + outs + inter + ws + draw
+
+
+def run_workload(args, cfg, world, rank, local_rank, dev, dist):
+    """Times one workload; returns the JSON line as a dict on rank 0 (None elsewhere)."""
     import paper_2509_05165_b200 as kvc
     from paper_2509_05165_b200 import workloads as W
     from paper_2509_05165_b200.binding import alloc_outputs
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-
-    cfg = rank_workload(pick_config(args), rank)
     wl = W.make_workload(cfg, dev)
     desc = kvc.desc_from_config(cfg)
     budget = cfg.budget
@@ -300,30 +354,46 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing
+    def timed(n):
+        """n passes back to back between two events; ms per pass, max over ranks."""
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(stream)
+        for _ in range(n):
+            step()
+        ev1.record(stream)
+        barrier()
+        return max_over_ranks([ev0.elapsed_time(ev1) / n], dist, dev)[0]
+
+    # ---- device-resident timing: exactly --steps passes (a burst of a few tens of milliseconds) ...
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
+    # (the clocks are sampled every 200 ms from before the first timed pass to after the last one of the
+    # long region: the --steps region alone is shorter than one sampling period)
     sampler = ClockSampler(gpu_id(local_rank)) if rank == 0 else None
+    if sampler:
+        time.sleep(0.3)                      # let the sampler come up before anything is timed
     kvc.kvc_launch_count(reset=True)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step()
-    ev1.record(stream)
-    barrier()
+    ms_per_step = timed(args.steps)
     launches = kvc.kvc_launch_count()
-    ms_total = ev0.elapsed_time(ev1)
     assert int(out.device_status.item()) == 0
+    # ---- ... and a long region (seconds: the clocks settle under the power cap)
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_long = max(args.steps, int(args.sustained_seconds * 1e3 / ms_per_step))
+        sustained = dict(steps=n_long, ms_per_step=timed(n_long))
+    clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["covers"] = "the %d-step region and the sustained region after it" % args.steps
 
     # ---- per-stage timing (the stage entry points, events between them)
     inter = alloc_outputs(desc, budget, wl.k[0].dtype, dev, keep_intermediates=True, workspace=out.workspace)
     names = ["score", "compose", "allocate", "gather"]
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     barrier()
-    for s in range(args.steps):
-        e = evs[s]
+    for st in range(args.steps):
+        e = evs[st]
         e[0].record(stream)
         kvc.kvc_score(desc, wl.q, wl.k, inter.scores, out.workspace, stream); e[1].record(stream)
         kvc.kvc_compose(desc, inter.scores, inter.idx, inter.composite, out.workspace, stream); e[2].record(stream)
@@ -332,7 +402,8 @@ def main():
         e[4].record(stream)
     barrier()
     stage_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / args.steps for i, n in enumerate(names)}
-    clocks = sampler.stop() if sampler else None
+    gpu_scores0 = inter.scores[0, 0].cpu().numpy() if rank == 0 else None       # layer 0, sequence 0
+    gpu_idx0 = inter.idx[0, 0].cpu().numpy() if rank == 0 else None
     del inter
 
     # ---- end to end: pinned host inputs -> device, pass, results -> pinned host
@@ -375,37 +446,105 @@ def main():
         del hq, hk, hv, h_kout, h_vout
 
     # ---- max over ranks
-    t = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0] + [stage_ms[n] for n in names], dist, dev)
-    ms_total, e2e_ms = t[0], t[1]
-    stage_ms = {n: t[2 + i] for i, n in enumerate(names)}
+    t = max_over_ranks([e2e["ms"] if e2e else 0.0] + [stage_ms[n] for n in names], dist, dev)
+    e2e_ms = t[0]
+    stage_ms = {n: t[1 + i] for i, n in enumerate(names)}
+    if rank != 0:
+        return None
 
-    if rank == 0:
-        ms_per_step = ms_total / args.steps
-        tokens = cfg.batch * cfg.n_ctx * world
-        value = aggregate_tokens_per_s(cfg, world, ms_per_step)
-        peak, peak_kind = measured_peaks()
-        ab = algorithmic_bytes(cfg)
-        dominant = max(("score", "gather"), key=lambda n: stage_ms[n])
-        ach = ab[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
-        line = dict(
-            metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
-            ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
-            dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
-            config=workload_config(cfg, world), clocks=clocks, gpu_launches=int(launches),
-            stage_ms=stage_ms,
-            pass_roofline=dict(bytes=ab["total"], achieved=ab["total"] / (ms_per_step * 1e-3) / 1e9, peak=peak,
-                               unit="GB/s", frac=ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
-                               peak_kind=peak_kind, frac_of_8tbs=ab["total"] / (ms_per_step * 1e-3) / 8e12),
-            roofline=dict(bound="hbm", kernel=dominant, achieved=ach, peak=peak, unit="GB/s", frac=ach / peak,
-                          traffic=SCORE_TRAFFIC_BYTES.get(cfg.name) if dominant == "score" else None,
-                          peak_kind=peak_kind, algorithmic_bytes=ab[dominant]),
-        )
-        if e2e:
-            line["e2e"] = dict(value=tokens / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=e2e["h2d"],
-                               d2h_bytes_per_step=e2e["d2h"], ms_per_step=e2e_ms, steps=e2e["steps"])
-        if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(cfg, args.cpu_seconds)
-        print(json.dumps(line))
+    tokens = cfg.batch * cfg.n_ctx * world
+    value = aggregate_tokens_per_s(cfg, world, ms_per_step)
+    peak, peak_kind = measured_peaks()
+    ab = algorithmic_bytes(cfg)
+    dominant = max(("score", "gather"), key=lambda n: stage_ms[n])
+    ach = ab[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
+
+    def pass_frac(ms):
+        return ab["total"] / (ms * 1e-3) / 1e9 / peak
+
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
+        config=workload_config(cfg, world), clocks=clocks, gpu_launches=int(launches),
+        stage_ms=stage_ms,
+        pass_roofline=dict(bytes=ab["total"], achieved=ab["total"] / (ms_per_step * 1e-3) / 1e9, peak=peak,
+                           unit="GB/s", frac=pass_frac(ms_per_step), peak_kind=peak_kind,
+                           frac_of_8tbs=ab["total"] / (ms_per_step * 1e-3) / 8e12,
+                           note="burst: %d passes back to back" % args.steps),
+        roofline=dict(bound="hbm", kernel=dominant, achieved=ach, peak=peak, unit="GB/s", frac=ach / peak,
+                      traffic=score_traffic_bytes(cfg) if dominant == "score" else None,
+                      peak_kind=peak_kind, algorithmic_bytes=ab[dominant]),
+    )
+    if sustained:
+        line["sustained"] = dict(steps=sustained["steps"], ms_per_step=sustained["ms_per_step"],
+                                 value=aggregate_tokens_per_s(cfg, world, sustained["ms_per_step"]),
+                                 pass_roofline_frac=pass_frac(sustained["ms_per_step"]))
+    if e2e:
+        line["e2e"] = dict(value=tokens / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=e2e["h2d"],
+                           d2h_bytes_per_step=e2e["d2h"], ms_per_step=e2e_ms, steps=e2e["steps"])
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(cfg, args.cpu_seconds)
+        line["parity"] = parity_summary(cfg, gpu_scores0, gpu_idx0)
+    return line
+
+
+SWEEP_N = (4096, 16384, 65536, 131072)
+SWEEP_BATCH = (1, 4, 8)
+SWEEP_RETENTION = (0.05, 0.10, 0.25, 0.50)
+
+
+def run_sweep(args, world, rank, local_rank, dev, dist):
+    """The N x batch x retention sweep on the 8B shape: one JSON line per point.  A point whose inputs,
+    outputs and workspace do not fit the free device memory is recorded as skipped, not attempted."""
+    from paper_2509_05165_b200 import workloads as W
+
+    args.no_e2e = True
+    args.no_cpu_baseline = True
+    args.sustained_seconds = 0.0
+    for n_ctx in SWEEP_N:
+        for batch in SWEEP_BATCH:
+            for ret in SWEEP_RETENTION:
+                cfg = rank_workload(W.sweep_config(n_ctx, batch, ret), rank)
+                free, _ = torch.cuda.mem_get_info()
+                need = device_bytes_needed(cfg)
+                fits = max_over_ranks([1.0 if need > 0.92 * free else 0.0], dist, dev)[0] == 0.0
+                if not fits:
+                    if rank == 0:
+                        print(json.dumps(dict(metric=METRIC, config=workload_config(cfg, world), value=None,
+                                              skipped="memory", bytes_needed=need, bytes_free=free)), flush=True)
+                    continue
+                line = run_workload(args, cfg, world, rank, local_rank, dev, dist)
+                if rank == 0:
+                    keep = ("metric", "value", "unit", "n_gpus", "steps", "ms_per_step", "config", "stage_ms", "pass_roofline")
+                    print(json.dumps({k: line[k] for k in keep}), flush=True)
+                torch.cuda.empty_cache()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    if args.sweep:
+        run_sweep(args, world, rank, local_rank, dev, dist)
+    else:
+        cfg = rank_workload(pick_config(args), rank)
+        line = run_workload(args, cfg, world, rank, local_rank, dev, dist)
+        if rank == 0:
+            print(json.dumps(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

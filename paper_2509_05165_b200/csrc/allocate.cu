@@ -112,15 +112,19 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
     // pooled index -> (row, position) once per tile, then by steps of the block width
     long long i = t0 + threadIdx.x;
     long long r = i / M, kk = i - r * M;
+    long long base = row_start(r, b, Bt, hpr, N) + floor;      // (recomputed only when the row changes)
 #pragma unroll 4
     for (int it = 0; it < kItemsPerThread; ++it) {
       if (i < total) {
-        const uint32_t key = score_to_key(composite[row_start(r, b, Bt, hpr, N) + floor + kk]);
+        const uint32_t key = score_to_key(composite[base + kk]);
         if ((key & hi_mask) == prefix) atomicAdd(&sh[(key >> shift) & 0xffu], 1u);
       }
       i += kHistThreads;
       kk += kHistThreads;
-      while (kk >= M) { kk -= M; ++r; }
+      if (kk >= M) {
+        while (kk >= M) { kk -= M; ++r; }
+        base = row_start(r, b, Bt, hpr, N) + floor;
+      }
     }
   }
   __syncthreads();

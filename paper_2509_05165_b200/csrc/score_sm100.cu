@@ -348,12 +348,17 @@ struct Cursor {
     b = lb - l * P.Bt;
   }
   // window rows of this unit's row tile (whole query heads; the last tile of a KV head may be short)
+  // (kLong: the instantiation that also handles windows longer than 128 rows, CH > 1; everywhere else
+  // that case is compiled out of the hot loops)
+  template <bool kLong>
   __device__ __forceinline__ int rows(const FastParams& P) const {
-    return P.CH == 1 ? min(P.HPT, P.G - q * P.HPT) * P.w : min(kRows, P.w - (q % P.CH) * kRows);
+    return (!kLong || P.CH == 1) ? min(P.HPT, P.G - q * P.HPT) * P.w : min(kRows, P.w - (q % P.CH) * kRows);
   }
   // first window row of this row tile inside its query head, and the tile's first query head in the group
-  __device__ __forceinline__ int row0(const FastParams& P) const { return P.CH == 1 ? 0 : (q % P.CH) * kRows; }
-  __device__ __forceinline__ int head0(const FastParams& P) const { return P.CH == 1 ? q * P.HPT : q / P.CH; }
+  template <bool kLong>
+  __device__ __forceinline__ int row0(const FastParams& P) const { return (!kLong || P.CH == 1) ? 0 : (q % P.CH) * kRows; }
+  template <bool kLong>
+  __device__ __forceinline__ int head0(const FastParams& P) const { return (!kLong || P.CH == 1) ? q * P.HPT : q / P.CH; }
   // index of the (layer, sequence, KV head)
   __device__ __forceinline__ int kv_unit(const FastParams& P) const { return (l * P.Bt + b) * P.Hkv + h; }
   __device__ __forceinline__ int tile(const FastParams& P) const { return j * P.RT + t; }
@@ -599,8 +604,9 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   }
   const int my_tiles = my_runs * P.RT;                  // stream length (some positions hold no tile)
   const int n_steps = my_tiles > 0 ? my_tiles + P.shift : 0;
+  constexpr bool kLong = (W == 0);   // only the run-time window variant has windows longer than 128 rows
   // the whole box arrives (rows outside the tensor as zeros)
-  const uint32_t q_bytes = (uint32_t)(P.CH == 1 ? P.HPT * P.w : kRows) * D * 2;
+  const uint32_t q_bytes = (uint32_t)((!kLong || P.CH == 1) ? P.HPT * P.w : kRows) * D * 2;
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
   if (warp == 0) {
@@ -638,7 +644,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
                 mbar_expect_tx(bar_qfull(qr.i), q_bytes);
                 for (int hf = 0; hf < SL::kHalves; ++hf)
                   tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
-                              bar_qfull(qr.i), hf * 64, c.row0(P), c.h * P.G + c.head0(P), c.b, pol_keep);
+                              bar_qfull(qr.i), hf * 64, c.template row0<kLong>(P), c.h * P.G + c.template head0<kLong>(P), c.b, pol_keep);
                 qr.next(kQSlots);
                 if (qc < kQSlots) ++qc;
               }
@@ -870,7 +876,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       if (!c.valid(P)) continue;
       const int tile = c.tile(P);
       const bool run_ends = c.last(P);
-      const bool row_used = row < c.rows(P);
+      const bool row_used = row < c.template rows<kLong>(P);
       if (c.t == 0 && half == 0) row_ref = __ldg(P.ref + (long long)c.u * kRows + row);   // used at the run's end
       const int buf = n1 & 1;
       // (the TMEM loads below are warp-wide instructions: the decision has to be the warp's)
@@ -893,7 +899,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           if (row_used) { fast_chunk(ra); fast_chunk(rb); }
         } else {
           float m2 = mref, l2 = lsum;                     // (the whole warp takes part in the TMEM loads)
-          const long long row_vis = min(P.N - 1, P.q_pos0 + (P.CH == 1 ? row_m : c.row0(P) + row));   // last key this row sees
+          const long long row_vis = min(P.N - 1, P.q_pos0 + ((!kLong || P.CH == 1) ? row_m : c.template row0<kLong>(P) + row));   // last key this row sees
           p1_masked_half(taddr, c0, row_vis, P.sl2e, &m2, &l2);
           if (row_used) { mref = m2; lsum = l2; }
           tc_fence_before();
@@ -944,6 +950,13 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     const unsigned long long scale2 = pack2(P.sl2e, P.sl2e);
     int n2 = 0;
     bool ok = true;
+    // per-tile work is kept to a minimum here: this group's instruction stream is what the kernel waits for
+    const bool gmax = P.agg_group == KVC_AGG_MAX;
+    const float inv_g = (P.QT == 1 && !gmax) ? 1.f / (float)P.G : 1.f;   // one row tile: the mean of Eq. 15 is finished here
+    const int vis_all_i = (int)vis_all;                // (N < 2^30)
+    const int n_ctx = (int)P.N;
+    int rows_u = 0, n_chunks = 0;                      // of the current run's unit
+    float* score_row = nullptr;                        // where that unit's scores (or partial aggregates) go
 
     Cursor cu;
     cu.init(P);
@@ -957,10 +970,11 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     }
     for (int idx = 0; idx < my_tiles; ++idx, cu.advance(P)) {
       if (!cu.valid(P)) continue;
-      const int tile = cu.tile(P);
-      const int rows_u = cu.rows(P);
-      const int n_chunks = (rows_u + 31) / 32;
+      const int tok0 = cu.tile(P) * kTile;             // first token of the tile
       if (cu.t == 0) {
+        rows_u = cu.template rows<kLong>(P);
+        n_chunks = (rows_u + 31) / 32;
+        score_row = P.scores + ((long long)cu.q * ((long long)P.L * P.Bt * P.Hkv) + cu.kv_unit(P)) * P.N;
         // a new run: its unit's log-sum-exp.  The short way: the row's pushed word, complete once
         // every run of the unit has arrived (fetched a tile or two ago; polled if it was not
         // complete then).  If a run's sum did not fit, the folded
@@ -1007,18 +1021,17 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       ++n2;
       if (!ok) continue;
       tc_fence_after();
-      const long long c = (long long)tile * kTile + trow;            // this thread's token
-      const bool full = (long long)tile * kTile + kTile - 1 <= vis_all;
+      const int c = tok0 + trow;                                     // this thread's token
+      const bool full = tok0 + kTile - 1 <= vis_all_i;
       float gacc;
       if (!kTaskMean && W >= 32 && full) {
         // the paper's default (max over the window) on a tile no mask touches: every 32-column
         // chunk belongs to one query head
-        gacc = (P.agg_group == KVC_AGG_MAX) ? -INFINITY : 0.f;
+        gacc = gmax ? -INFINITY : 0.f;
         float hacc = -INFINITY;
         uint32_t r[32];
         tc_ld32_nowait(lane_addr + tmem_col, r);
-#pragma unroll 1
-        for (int j = 0; j < n_chunks; ++j) {
+        auto chunk = [&](const int j, const bool last) {
           // the rows' -log-sum-exp for this chunk, fetched while the accumulator load is in flight
           ulonglong2 nl[8];
           {
@@ -1035,7 +1048,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             unpack2(y0, x[4 * i], x[4 * i + 1]);                     // log2 of the attention weights
             unpack2(y1, x[4 * i + 2], x[4 * i + 3]);
           }
-          if (j + 1 < n_chunks) {
+          if (!last) {
             tc_ld32_nowait(lane_addr + tmem_col + (j + 1) * 32, r);
           } else {
             tc_fence_before();                                        // the accumulator has been read
@@ -1049,29 +1062,29 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
           hacc = max3(hacc, x[30], x[31]);
           if (((j + 1) * 32) % (W > 0 ? W : 1) == 0) {
             const float s_task = ex2(hacc);
-            gacc = (P.agg_group == KVC_AGG_MAX) ? fmaxf(gacc, s_task) : gacc + s_task;
+            gacc = gmax ? fmaxf(gacc, s_task) : gacc + s_task;
             hacc = -INFINITY;
           }
-        }
+        };
+#pragma unroll 1
+        for (int j = 0; j < n_chunks; ++j) chunk(j, j + 1 == n_chunks);
       } else if (W == 0 && P.CH > 1) {
         // a window longer than 128 rows: the tile holds rows row0 .. of one query head and yields
         // that head's partial Eq. 14 (the maximum, or the sum, over these rows)
         gacc = p2_long_tile<kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
-                                       c - P.q_pos0 - cu.row0(P));
+                                       (long long)c - P.q_pos0 - cu.template row0<kLong>(P));
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(buf));
       } else {
         gacc = p2_generic_tile<W, kTaskMean>(lane_addr + tmem_col, neg_lse, n_chunks, rows_u, P.sl2e, full,
-                                             c - P.q_pos0, P.agg_group, P.w);
+                                             (long long)c - P.q_pos0, P.agg_group, P.w);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(buf));
       }
       // one row tile: the group aggregate itself; several: this tile's part of it
-      if (P.QT == 1 && P.agg_group == KVC_AGG_MEAN) gacc = gacc / (float)P.G;
-      if (c < P.N)
-        P.scores[((long long)cu.q * ((long long)P.L * P.Bt * P.Hkv) + cu.kv_unit(P)) * P.N + c] = gacc;
+      if (c < n_ctx) score_row[c] = gacc * inv_g;
     }
   }
 
