@@ -278,6 +278,26 @@ KVC_API kvc_status kvc_compress_unstructured(const kvc_desc* desc, const void* c
                                      float* scores_out, int32_t* device_status, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
+/*
+ * Support for sharding ONE sequence's KV heads over several GPUs (tensor-parallel serving).  Scoring
+ * and ranking are per head and stay local; two steps need the other ranks' heads: the head-mean term
+ * of Eq. 16 and the aggregation over heads of Eq. 19.  With desc describing the LOCAL heads (and
+ * augment_head_mean = 0 for kvc_score, so that it returns the group aggregates of Eq. 15):
+ *   kvc_head_sum:      head_sum[l, b, c] = sum over the local KV heads of scores[l, b, h, c]
+ *                      -- the caller all-reduces (sum) head_sum over the ranks --
+ *   kvc_add_head_mean: scores[l, b, h, c] += head_sum[l, b, c] / n_kv_heads_total            (Eq. 16)
+ *   kvc_compose on the local heads gives the local mean (or max) of Eq. 19; the caller all-reduces it
+ *   (sum, then kvc_scale by 1 / ranks for equal shards; max for KVC_AGG_MAX); kvc_allocate then runs
+ *   replicated on identical inputs and kvc_gather on the local heads.
+ * The paper has no multi-GPU formulation; the sums are the same terms in another order, so scores and
+ * composite scores agree with the single-GPU pass to fp32 rounding, not bit for bit.
+ * scores: [L, batch, Hkv_local, N]; head_sum: [L, batch, N]; x: n floats.  No workspace needed.
+ */
+KVC_API kvc_status kvc_head_sum(const kvc_desc* desc, const float* scores, float* head_sum, void* stream);
+KVC_API kvc_status kvc_add_head_mean(const kvc_desc* desc, float* scores, const float* head_sum,
+                             int32_t n_kv_heads_total, void* stream);
+KVC_API kvc_status kvc_scale(float* x, int64_t n, float factor, void* stream);
+
 /* Message of the last error returned on this thread (static storage; never NULL). */
 KVC_API const char* kvc_last_error(void);
 

@@ -84,6 +84,12 @@ def _load():
     lib.kvc_gather_unstructured.restype = C.c_int
     lib.kvc_compress_unstructured.argtypes = [dp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.kvc_compress_unstructured.restype = C.c_int
+    lib.kvc_head_sum.argtypes = [dp, vp, vp, vp]
+    lib.kvc_head_sum.restype = C.c_int
+    lib.kvc_add_head_mean.argtypes = [dp, vp, vp, i32, vp]
+    lib.kvc_add_head_mean.restype = C.c_int
+    lib.kvc_scale.argtypes = [vp, i64, C.c_float, vp]
+    lib.kvc_scale.restype = C.c_int
     lib.kvc_compose.argtypes = [dp, vp, vp, vp, vp, sz, vp]
     lib.kvc_compose.restype = C.c_int
     lib.kvc_allocate.argtypes = [dp, vp, i64, vp, vp, vp, sz, vp]
@@ -181,6 +187,19 @@ def kvc_debug_score_hooks(wait_limit_ns: int = 0, withhold_unit: int = -1) -> No
     """Test hook: bound of the scoring kernel's device-side waits, and a unit whose statistics
     are withheld so that those waits expire.  The defaults restore normal operation."""
     _load().kvc_debug_score_hooks(int(wait_limit_ns), int(withhold_unit))
+
+
+def kvc_head_sum(desc, scores, head_sum, stream=None) -> None:
+    _check(_load().kvc_head_sum(C.byref(desc), _dptr(scores), _dptr(head_sum), _stream(stream)))
+
+
+def kvc_add_head_mean(desc, scores, head_sum, n_kv_heads_total: int, stream=None) -> None:
+    _check(_load().kvc_add_head_mean(C.byref(desc), _dptr(scores), _dptr(head_sum), int(n_kv_heads_total),
+                                     _stream(stream)))
+
+
+def kvc_scale(x: torch.Tensor, factor: float, stream=None) -> None:
+    _check(_load().kvc_scale(_dptr(x), x.numel(), float(factor), _stream(stream)))
 
 
 def kvc_compose(desc, scores, idx, composite, workspace, stream=None) -> None:

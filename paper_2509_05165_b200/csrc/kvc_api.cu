@@ -521,6 +521,33 @@ kvc_status kvc_compress_unstructured(const kvc_desc* d, const void* const* q, co
                        k_out, v_out, st);
 }
 
+kvc_status kvc_head_sum(const kvc_desc* d, const float* scores, float* head_sum, void* stream) {
+  Problem P; GroupMap gm;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  KVC_REQUIRE(scores && head_sum, KVC_ERR_INVALID_ARG, "scores or head_sum is NULL");
+  if ((s = check_device()) != KVC_OK) return s;
+  return launch_head_sum(P, scores, head_sum, (cudaStream_t)stream);
+}
+
+kvc_status kvc_add_head_mean(const kvc_desc* d, float* scores, const float* head_sum, int32_t n_kv_heads_total,
+                             void* stream) {
+  Problem P; GroupMap gm;
+  kvc_status s;
+  if ((s = resolve(d, &P, &gm)) != KVC_OK) return s;
+  KVC_REQUIRE(scores && head_sum, KVC_ERR_INVALID_ARG, "scores or head_sum is NULL");
+  KVC_REQUIRE(n_kv_heads_total >= P.Hkv, KVC_ERR_INVALID_ARG, "n_kv_heads_total is smaller than the local head count");
+  if ((s = check_device()) != KVC_OK) return s;
+  return launch_add_head_mean(P, scores, head_sum, n_kv_heads_total, (cudaStream_t)stream);
+}
+
+kvc_status kvc_scale(float* x, int64_t n, float factor, void* stream) {
+  KVC_REQUIRE(x != nullptr && n >= 0, KVC_ERR_INVALID_ARG, "x is NULL or n < 0");
+  kvc_status s;
+  if ((s = check_device()) != KVC_OK) return s;
+  return launch_scale(x, n, factor, (cudaStream_t)stream);
+}
+
 const char* kvc_last_error(void) { return g_err; }
 
 int64_t kvc_launch_count(int32_t reset) {

@@ -147,6 +147,10 @@ kvc_status launch_gather(const Problem& P, const LayerPtrs& k, const LayerPtrs& 
 // ---- variants ---------------------------------------------------------------------------------
 // ||v||_2 of every value row in fp32: vnorm [L, Bt, Hkv, N] (App. A.1.3).
 kvc_status launch_value_norm(const Problem& P, const LayerPtrs& v, float* vnorm, cudaStream_t st);
+// Head-sharded scoring (see kvc.h).
+kvc_status launch_head_sum(const Problem& P, const float* scores, float* head_sum, cudaStream_t st);
+kvc_status launch_add_head_mean(const Problem& P, float* scores, const float* head_sum, int heads_total, cudaStream_t st);
+kvc_status launch_scale(float* x, long long n, float f, cudaStream_t st);
 // The first n_keep entries of every idx row in ascending position, in place.  n_keep per layer
 // [Bt, L] or, per_head, per (layer, head) [Bt, L * Hkv].
 size_t order_kept_workspace_bytes(const Problem& P);

@@ -99,7 +99,61 @@ order_kept_kernel(int32_t* __restrict__ idx, const int32_t* __restrict__ n_keep,
   }
 }
 
+// Head-sharded scoring: the local part of Eq. 16's sum over the KV heads, and the mean added back.
+__global__ void head_sum_kernel(const float* __restrict__ s, float* __restrict__ head_sum, int Hkv, long long N,
+                                long long total) {
+  grid_dependency_wait();
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const long long lb = i / N, c = i - lb * N;
+  const float* base = s + lb * Hkv * N + c;
+  float sum = 0.f;
+  for (int h = 0; h < Hkv; ++h) sum += base[(long long)h * N];
+  head_sum[i] = sum;
+}
+
+__global__ void add_head_mean_kernel(float* __restrict__ s, const float* __restrict__ head_sum, int Hkv, float inv_total,
+                                     long long N, long long total) {
+  grid_dependency_wait();
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const long long lb = i / N, c = i - lb * N;
+  float* base = s + lb * Hkv * N + c;
+  const float mean = head_sum[i] * inv_total;
+  for (int h = 0; h < Hkv; ++h) base[(long long)h * N] += mean;
+}
+
+__global__ void scale_kernel(float* __restrict__ x, long long n, float f) {
+  grid_dependency_wait();
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) x[i] *= f;
+}
+
 }  // namespace
+
+kvc_status launch_head_sum(const Problem& P, const float* scores, float* head_sum, cudaStream_t st) {
+  const long long total = (long long)P.L * P.Bt * P.N;
+  KVC_CUDA(launch_dependent(head_sum_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, scores, head_sum,
+                            P.Hkv, P.N, total));
+  KVC_LAUNCH_CHECK("head_sum_kernel");
+  return KVC_OK;
+}
+
+kvc_status launch_add_head_mean(const Problem& P, float* scores, const float* head_sum, int heads_total,
+                                cudaStream_t st) {
+  const long long total = (long long)P.L * P.Bt * P.N;
+  KVC_CUDA(launch_dependent(add_head_mean_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, scores,
+                            head_sum, P.Hkv, 1.0f / (float)heads_total, P.N, total));
+  KVC_LAUNCH_CHECK("add_head_mean_kernel");
+  return KVC_OK;
+}
+
+kvc_status launch_scale(float* x, long long n, float f, cudaStream_t st) {
+  if (n <= 0) return KVC_OK;
+  KVC_CUDA(launch_dependent(scale_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, x, n, f));
+  KVC_LAUNCH_CHECK("scale_kernel");
+  return KVC_OK;
+}
 
 kvc_status launch_value_norm(const Problem& P, const LayerPtrs& v, float* vnorm, cudaStream_t st) {
   const long long rows = (long long)P.L * P.Bt * P.Hkv * P.N;
