@@ -204,8 +204,10 @@ KVC_API kvc_status kvc_order_kept(const kvc_desc* desc, int32_t* idx, const int3
  * afterwards (the call synchronises the device and can fail once memory is fragmented), or a
  * plug-in that is handed the host application's tensors but no allocator.  The scratch of the
  * selection lives instead in a fixed array inside the library image: 256 KiB of device memory on
- * every GPU that loads the library, held until the process exits.  The call allocates and frees
- * nothing, on the device or through any library.
+ * every GPU that loads the library, held until the process exits.  The call itself calls no
+ * allocator, on the device or through any library.  One thing to plan for: with CUDA's lazy module
+ * loading the array is reserved on a device when the library's code is first used there, which can
+ * be this entry point's first call on that device -- so make that first call during start-up.
  *
  *   - desc->batch must be <= KVC_STATIC_MAX_BATCH; a larger batch returns KVC_ERR_UNSUPPORTED
  *     and launches nothing.

@@ -48,6 +48,32 @@ def test_static_scratch_allocation_matches_workspace_allocation_twice():
         assert n_got.sum(dim=1).tolist() == [budget] * Bt
 
 
+@pytest.mark.gpu
+def test_static_scratch_at_its_largest_batch_and_on_a_side_stream():
+    """64 sequences use the whole built-in array; a call on another stream than the default one
+    gives the same result as long as nothing else that uses the array overlaps it."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    dev = torch.device("cuda:0")
+    L, Bt, N = 3, 64, 300
+    desc = kvc.kvc_desc_init(L, Bt, 4, 2, 64, N, 8, kvc.BF16)
+    ws = torch.empty(kvc.kvc_workspace_size(desc, 0), dtype=torch.uint8, device=dev)
+    side = torch.cuda.Stream(dev)
+    for seed, budget, stream in ((5, 401, None), (6, 77, side), (7, 640, side)):
+        I = _composite(L, Bt, N, seed, dev)
+        n_ref = torch.empty((Bt, L), dtype=torch.int32, device=dev)
+        off_ref = torch.empty((Bt, L + 1), dtype=torch.int64, device=dev)
+        kvc.kvc_allocate(desc, I, budget, n_ref, off_ref, ws)
+        torch.cuda.synchronize()                     # the side stream must not start before I and the reference are there
+        n_got = torch.full((Bt, L), -7, dtype=torch.int32, device=dev)
+        off_got = torch.full((Bt, L + 1), -7, dtype=torch.int64, device=dev)
+        torch.cuda.synchronize()
+        kvc.kvc_allocate_static(desc, I, budget, n_got, off_got, stream)
+        torch.cuda.synchronize()
+        assert torch.equal(n_got, n_ref) and torch.equal(off_got, off_ref), (seed, budget)
+        assert n_got.sum(dim=1).tolist() == [budget] * Bt
+
+
 def test_static_scratch_allocation_rejects_a_batch_beyond_its_maximum():
     """Host-side check, no launch: the fixed array covers 64 sequences."""
     desc = kvc.kvc_desc_init(2, 65, 4, 2, 64, 128, 8, kvc.BF16)
