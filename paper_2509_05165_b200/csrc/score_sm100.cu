@@ -609,224 +609,9 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
   const uint32_t q_bytes = (uint32_t)((!kLong || P.CH == 1) ? P.HPT * P.w : kRows) * D * 2;
   const long long vis_all = min(P.N - 1, P.q_pos0);          // tokens up to here are seen by every row
 
-  if (warp == 0) {
-    // ============================== TMA producer ==============================================
-    if (lane == 0) {
-      unsigned long long pol_stream, pol_keep;
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-      Ring kr = {0, 0}, qr = {0, 0};   // next K stage / Q slot to fill; phase = parity of the fill count / ring size
-      int nk = 0, qc = 0;              // K tiles / Q tiles issued (saturating small counts are all that is needed)
-      bool ok = true;
-      Cursor cur[2], ahead;            // the two streams, and the pass-1 stream kPrefetch tiles ahead
-      cur[0].init(P); cur[1].init(P); ahead.init(P);
-      int ahead_pos = 0;
-      auto prefetch_next = [&]() {
-        if (ahead_pos >= my_tiles) return;
-        if (ahead.valid(P)) {
-          for (int hf = 0; hf < SL::kHalves; ++hf)
-            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile(P) * kTile, ahead.h, ahead.b);
-        }
-        ahead.advance(P);
-        ++ahead_pos;
-      };
-      for (int i = 0; i < kPrefetch; ++i) prefetch_next();
-      for (int i = 0; i < n_steps && ok; ++i) {
-#pragma unroll
-        for (int pass = 0; pass < 2; ++pass) {
-          const int idx = pass == 0 ? i : i - P.shift;
-          if (!ok || idx < 0 || idx >= my_tiles) continue;
-          Cursor& c = cur[pass];
-          if (c.valid(P)) {
-            if (c.t == 0) {                                    // a new run: its Q goes into the next ring slot
-              if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), ctl);
-              if (ok) {
-                mbar_expect_tx(bar_qfull(qr.i), q_bytes);
-                for (int hf = 0; hf < SL::kHalves; ++hf)
-                  tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
-                              bar_qfull(qr.i), hf * 64, c.template row0<kLong>(P), c.h * P.G + c.template head0<kLong>(P), c.b, pol_keep);
-                qr.next(kQSlots);
-                if (qc < kQSlots) ++qc;
-              }
-            }
-            if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), ctl);
-            if (ok) {
-              mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
-              // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
-              for (int hf = 0; hf < SL::kHalves; ++hf)
-                tma_load_4d(sbase + SL::kK + kr.i * SL::kTileBytes + hf * (kTile * 128), P.k_maps + c.l,
-                            bar_kfull(kr.i), hf * 64, c.tile(P) * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
-              kr.next(SL::kStages);
-              if (nk < SL::kStages) ++nk;
-            }
-          }
-          c.advance(P);
-          if (pass == 0) prefetch_next();
-        }
-      }
-      // drain: every issued copy must have landed before the CTA's shared memory is released
-      // (an issued copy always completes, so these waits do not take the abort shortcut).
-      // The last fill of stage i is complete once its full barrier has left the phase of that fill.
-      for (int n = 0; n < nk; ++n) {
-        // walk the ring backwards from the slot before kr
-        int i2 = kr.i - 1 - n, ph = kr.phase;
-        if (i2 < 0) { i2 += SL::kStages; ph ^= 1; }
-        mbar_wait_issued(bar_kfull(i2), (uint32_t)ph, ctl);
-      }
-      for (int n = 0; n < qc; ++n) {
-        int i2 = qr.i - 1 - n, ph = qr.phase;
-        if (i2 < 0) { i2 += kQSlots; ph ^= 1; }
-        mbar_wait_issued(bar_qfull(i2), (uint32_t)ph, ctl);
-      }
-    }
-  } else if (warp < 3) {
-    // ============================== MMA issuers ================================================
-    // Both walk the whole sequence (the rings are shared and filled in sequence order) and each
-    // issues the tiles of its own pass.  Each also waits for the fills that belong to the other
-    // pass and acknowledges them: a parity wait is only meaningful for the phase that follows the
-    // last one seen, so neither thread may skip a phase of a ring barrier, and the producer must
-    // not refill a slot before both have seen its fill (the "empty" barriers count two arrivals:
-    // the user's commit and the other thread's acknowledgement).
-    if (lane == 0) {
-      const int mine = warp - 1;       // the pass this thread issues
-      Ring kr = {0, 0}, qr = {0, 0};
-      Ring tb = {0, 0};                // accumulator buffer of this pass (two per pass)
-      int nt = 0;                      // tiles issued (saturating at 2)
-      int cur_slot = 0;
-      bool ok = true;
-      Cursor cur[2];
-      cur[0].init(P); cur[1].init(P);
-      for (int i = 0; i < n_steps && ok; ++i) {
-#pragma unroll
-        for (int pass = 0; pass < 2; ++pass) {
-          const int idx = pass == 0 ? i : i - P.shift;
-          if (!ok || idx < 0 || idx >= my_tiles) continue;
-          Cursor& c = cur[pass];
-          if (c.valid(P)) {
-            if (c.t == 0) {
-              ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, ctl);
-              if (pass == mine) cur_slot = qr.i;
-              else if (ok) mbar_arrive(bar_qfree(qr.i));
-            }
-            if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, ctl);
-            if (ok && pass != mine) mbar_arrive(bar_kempty(kr.i));
-            if (pass == mine) {
-              const int buf = pass * 2 + tb.i;
-              if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), ctl);
-              if (ok) {
-                tc_fence_after();
-                const uint64_t dq0 = umma_desc(sbase + SL::kQ + cur_slot * SL::kTileBytes);
-                const uint64_t dk0 = umma_desc(sbase + SL::kK + kr.i * SL::kTileBytes);
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                  // the start-address field counts 16-byte units: 64-element half, then 32 B per K step
-                  const uint64_t off = (uint64_t)(((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4);
-                  // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
-                  if (pass == 0) tc_mma_bf16(d_tmem, dq0 + off, dk0 + off, kIdesc, kk > 0);
-                  else tc_mma_bf16(d_tmem, dk0 + off, dq0 + off, kIdesc, kk > 0);
-                }
-                tc_commit(bar_kempty(kr.i));   // the K stage may be refilled once these MMAs are done
-                tc_commit(bar_tfull(buf));     // ... and the accumulator is then complete
-                if (c.last(P)) tc_commit(bar_qfree(cur_slot));
-                tb.next(2);
-                if (nt < 2) ++nt;
-              }
-            }
-            if (c.t == 0) qr.next(kQSlots);
-            kr.next(SL::kStages);
-          }
-          c.advance(P);
-        }
-      }
-      // no MMA may be in flight when the TMEM columns and the shared memory are given back
-      if (nt > 0) {
-        tc_commit(bar_mma_done(mine));
-        mbar_wait_issued(bar_mma_done(mine), 0u, ctl);
-      }
-    }
-  } else if (warp == 3) {
-    // ============================== statistics exchange ========================================
-    // This CTA folds the groups  x, x + grid, ...  (x = blockIdx.x; a group is numbered
-    // unit * NG + group) and the units  x, x + grid, ...   Jobs are taken in the order in which
-    // they become ready anywhere in the grid -- a group before every unit whose last group is
-    // not smaller -- so a wait here only ever depends on jobs that are earlier in that order.
-    // Lane i owns rows 4i .. 4i+3; a record of 128 rows is 64 float4, two per lane.
-    const int n_groups = P.U * P.NG;
-    int gi = blockIdx.x, un = blockIdx.x;             // next group / next unit of this CTA
-    bool ok = my_runs > 0;
-    while (ok && (gi < n_groups || un < P.U)) {
-      const bool take_group = gi < n_groups && (un >= P.U || gi <= (un + 1) * P.NG - 1);
-      const int* counter = take_group ? P.group_counter + gi : P.unit_counter + un;
-      int target;                                     // the counters start at -1
-      if (take_group) {
-        const int g = gi % P.NG;
-        target = min(kGroupRuns, P.RPU - g * kGroupRuns) - 1;
-      } else {
-        target = P.NG - 1;
-      }
-      if (lane == 0) {
-        const unsigned long long t0 = globaltimer_ns();
-        uint32_t spins = 0;
-        while (ld_acquire_s32(counter) != target) {
-          __nanosleep(200);
-          if ((++spins & 63u) == 0 && give_up(ctl, t0)) { ok = false; break; }
-        }
-      }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-      __threadfence();                                // the records were published before the counts we saw
-      float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
-      if (take_group) {
-        const int u = gi / P.NG, g = gi - u * P.NG;
-        const int members = target + 1;
-        const float4* src = P.partial + ((long long)u * P.RPU + g * kGroupRuns) * 64 + 2 * lane;
-        // four records in flight at a time (this warp runs on a small register budget)
-#pragma unroll 1
-        for (int r0 = 0; r0 < members; r0 += 4) {
-          float4 v[8];
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            if (r0 + r < members) { v[2 * r] = __ldcg(src + (r0 + r) * 64); v[2 * r + 1] = __ldcg(src + (r0 + r) * 64 + 1); }
-          }
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            if (r0 + r < members) {
-              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
-              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
-              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
-              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
-            }
-          }
-        }
-        float4* dst = P.group_partial + (long long)gi * 64 + 2 * lane;
-        dst[0] = lo;
-        dst[1] = hi;
-        __syncwarp();
-        if (lane == 0) {
-          __threadfence();
-          red_add_release(P.unit_counter + u, 1);
-        }
-        gi += P.grid;
-      } else {
-        const float4* src = P.group_partial + (long long)un * P.NG * 64 + 2 * lane;
-#pragma unroll 2
-        for (int r = 0; r < P.NG; ++r) {
-          const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
-          combine(lo.x, lo.y, v0.x, v0.y);
-          combine(lo.z, lo.w, v0.z, v0.w);
-          combine(hi.x, hi.y, v1.x, v1.y);
-          combine(hi.z, hi.w, v1.z, v1.w);
-        }
-        unsigned int* out = P.lse2 + (long long)un * kRows + 4 * lane;
-        st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
-        st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
-        st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
-        st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
-        un += P.grid;
-      }
-    }
-  } else if (warp >= 8) {
+  // (The order of the roles in the code is not neutral: their hot loops share the instruction caches,
+  // and this order measured fastest.)
+  if (warp >= 8) {
     // ============================== pass-1 epilogue ============================================
     const int half = (warp - 8) >> 2;                 // which 64 columns (tokens) of every tile
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
@@ -941,7 +726,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         mref = -INFINITY; lsum = 0.f;
       }
     }
-  } else {
+  } else if (warp >= 4 && warp < 8) {
     // ============================== pass-2 epilogue ============================================
     const int quarter = warp & 3;
     const int trow = quarter * 32 + lane;             // TMEM lane = token inside the tile; also 0..127 in the group
@@ -1085,6 +870,223 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       }
       // one row tile: the group aggregate itself; several: this tile's part of it
       if (c < n_ctx) score_row[c] = gacc * inv_g;
+    }
+  } else if (warp == 1 || warp == 2) {
+    // ============================== MMA issuers ================================================
+    // Both walk the whole sequence (the rings are shared and filled in sequence order) and each
+    // issues the tiles of its own pass.  Each also waits for the fills that belong to the other
+    // pass and acknowledges them: a parity wait is only meaningful for the phase that follows the
+    // last one seen, so neither thread may skip a phase of a ring barrier, and the producer must
+    // not refill a slot before both have seen its fill (the "empty" barriers count two arrivals:
+    // the user's commit and the other thread's acknowledgement).
+    if (lane == 0) {
+      const int mine = warp - 1;       // the pass this thread issues
+      Ring kr = {0, 0}, qr = {0, 0};
+      Ring tb = {0, 0};                // accumulator buffer of this pass (two per pass)
+      int nt = 0;                      // tiles issued (saturating at 2)
+      int cur_slot = 0;
+      bool ok = true;
+      Cursor cur[2];
+      cur[0].init(P); cur[1].init(P);
+      for (int i = 0; i < n_steps && ok; ++i) {
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+          const int idx = pass == 0 ? i : i - P.shift;
+          if (!ok || idx < 0 || idx >= my_tiles) continue;
+          Cursor& c = cur[pass];
+          if (c.valid(P)) {
+            if (c.t == 0) {
+              ok = mbar_wait(bar_qfull(qr.i), (uint32_t)qr.phase, ctl);
+              if (pass == mine) cur_slot = qr.i;
+              else if (ok) mbar_arrive(bar_qfree(qr.i));
+            }
+            if (ok) ok = mbar_wait(bar_kfull(kr.i), (uint32_t)kr.phase, ctl);
+            if (ok && pass != mine) mbar_arrive(bar_kempty(kr.i));
+            if (pass == mine) {
+              const int buf = pass * 2 + tb.i;
+              if (ok && nt >= 2) ok = mbar_wait(bar_tempty(buf), (uint32_t)(tb.phase ^ 1), ctl);
+              if (ok) {
+                tc_fence_after();
+                const uint64_t dq0 = umma_desc(sbase + SL::kQ + cur_slot * SL::kTileBytes);
+                const uint64_t dk0 = umma_desc(sbase + SL::kK + kr.i * SL::kTileBytes);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTile;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                  // the start-address field counts 16-byte units: 64-element half, then 32 B per K step
+                  const uint64_t off = (uint64_t)(((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4);
+                  // pass 1: rows = query rows (A = Q), columns = tokens (B = K); pass 2: swapped
+                  if (pass == 0) tc_mma_bf16(d_tmem, dq0 + off, dk0 + off, kIdesc, kk > 0);
+                  else tc_mma_bf16(d_tmem, dk0 + off, dq0 + off, kIdesc, kk > 0);
+                }
+                tc_commit(bar_kempty(kr.i));   // the K stage may be refilled once these MMAs are done
+                tc_commit(bar_tfull(buf));     // ... and the accumulator is then complete
+                if (c.last(P)) tc_commit(bar_qfree(cur_slot));
+                tb.next(2);
+                if (nt < 2) ++nt;
+              }
+            }
+            if (c.t == 0) qr.next(kQSlots);
+            kr.next(SL::kStages);
+          }
+          c.advance(P);
+        }
+      }
+      // no MMA may be in flight when the TMEM columns and the shared memory are given back
+      if (nt > 0) {
+        tc_commit(bar_mma_done(mine));
+        mbar_wait_issued(bar_mma_done(mine), 0u, ctl);
+      }
+    }
+  } else if (warp == 0) {
+    // ============================== TMA producer ==============================================
+    if (lane == 0) {
+      unsigned long long pol_stream, pol_keep;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+      Ring kr = {0, 0}, qr = {0, 0};   // next K stage / Q slot to fill; phase = parity of the fill count / ring size
+      int nk = 0, qc = 0;              // K tiles / Q tiles issued (saturating small counts are all that is needed)
+      bool ok = true;
+      Cursor cur[2], ahead;            // the two streams, and the pass-1 stream kPrefetch tiles ahead
+      cur[0].init(P); cur[1].init(P); ahead.init(P);
+      int ahead_pos = 0;
+      auto prefetch_next = [&]() {
+        if (ahead_pos >= my_tiles) return;
+        if (ahead.valid(P)) {
+          for (int hf = 0; hf < SL::kHalves; ++hf)
+            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile(P) * kTile, ahead.h, ahead.b);
+        }
+        ahead.advance(P);
+        ++ahead_pos;
+      };
+      for (int i = 0; i < kPrefetch; ++i) prefetch_next();
+      for (int i = 0; i < n_steps && ok; ++i) {
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+          const int idx = pass == 0 ? i : i - P.shift;
+          if (!ok || idx < 0 || idx >= my_tiles) continue;
+          Cursor& c = cur[pass];
+          if (c.valid(P)) {
+            if (c.t == 0) {                                    // a new run: its Q goes into the next ring slot
+              if (qc >= kQSlots) ok = mbar_wait(bar_qfree(qr.i), (uint32_t)(qr.phase ^ 1), ctl);
+              if (ok) {
+                mbar_expect_tx(bar_qfull(qr.i), q_bytes);
+                for (int hf = 0; hf < SL::kHalves; ++hf)
+                  tma_load_4d(sbase + SL::kQ + qr.i * SL::kTileBytes + hf * (kTile * 128), P.q_maps + c.l,
+                              bar_qfull(qr.i), hf * 64, c.template row0<kLong>(P), c.h * P.G + c.template head0<kLong>(P), c.b, pol_keep);
+                qr.next(kQSlots);
+                if (qc < kQSlots) ++qc;
+              }
+            }
+            if (ok && nk >= SL::kStages) ok = mbar_wait(bar_kempty(kr.i), (uint32_t)(kr.phase ^ 1), ctl);
+            if (ok) {
+              mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
+              // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
+              for (int hf = 0; hf < SL::kHalves; ++hf)
+                tma_load_4d(sbase + SL::kK + kr.i * SL::kTileBytes + hf * (kTile * 128), P.k_maps + c.l,
+                            bar_kfull(kr.i), hf * 64, c.tile(P) * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
+              kr.next(SL::kStages);
+              if (nk < SL::kStages) ++nk;
+            }
+          }
+          c.advance(P);
+          if (pass == 0) prefetch_next();
+        }
+      }
+      // drain: every issued copy must have landed before the CTA's shared memory is released
+      // (an issued copy always completes, so these waits do not take the abort shortcut).
+      // The last fill of stage i is complete once its full barrier has left the phase of that fill.
+      for (int n = 0; n < nk; ++n) {
+        // walk the ring backwards from the slot before kr
+        int i2 = kr.i - 1 - n, ph = kr.phase;
+        if (i2 < 0) { i2 += SL::kStages; ph ^= 1; }
+        mbar_wait_issued(bar_kfull(i2), (uint32_t)ph, ctl);
+      }
+      for (int n = 0; n < qc; ++n) {
+        int i2 = qr.i - 1 - n, ph = qr.phase;
+        if (i2 < 0) { i2 += kQSlots; ph ^= 1; }
+        mbar_wait_issued(bar_qfull(i2), (uint32_t)ph, ctl);
+      }
+    }
+  } else if (warp == 3) {
+    // ============================== statistics exchange ========================================
+    // This CTA folds the groups  x, x + grid, ...  (x = blockIdx.x; a group is numbered
+    // unit * NG + group) and the units  x, x + grid, ...   Jobs are taken in the order in which
+    // they become ready anywhere in the grid -- a group before every unit whose last group is
+    // not smaller -- so a wait here only ever depends on jobs that are earlier in that order.
+    // Lane i owns rows 4i .. 4i+3; a record of 128 rows is 64 float4, two per lane.
+    const int n_groups = P.U * P.NG;
+    int gi = blockIdx.x, un = blockIdx.x;             // next group / next unit of this CTA
+    bool ok = my_runs > 0;
+    while (ok && (gi < n_groups || un < P.U)) {
+      const bool take_group = gi < n_groups && (un >= P.U || gi <= (un + 1) * P.NG - 1);
+      const int* counter = take_group ? P.group_counter + gi : P.unit_counter + un;
+      int target;                                     // the counters start at -1
+      if (take_group) {
+        const int g = gi % P.NG;
+        target = min(kGroupRuns, P.RPU - g * kGroupRuns) - 1;
+      } else {
+        target = P.NG - 1;
+      }
+      if (lane == 0) {
+        const unsigned long long t0 = globaltimer_ns();
+        uint32_t spins = 0;
+        while (ld_acquire_s32(counter) != target) {
+          __nanosleep(200);
+          if ((++spins & 63u) == 0 && give_up(ctl, t0)) { ok = false; break; }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      __threadfence();                                // the records were published before the counts we saw
+      float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
+      if (take_group) {
+        const int u = gi / P.NG, g = gi - u * P.NG;
+        const int members = target + 1;
+        const float4* src = P.partial + ((long long)u * P.RPU + g * kGroupRuns) * 64 + 2 * lane;
+        // four records in flight at a time (this warp runs on a small register budget)
+#pragma unroll 1
+        for (int r0 = 0; r0 < members; r0 += 4) {
+          float4 v[8];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            if (r0 + r < members) { v[2 * r] = __ldcg(src + (r0 + r) * 64); v[2 * r + 1] = __ldcg(src + (r0 + r) * 64 + 1); }
+          }
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            if (r0 + r < members) {
+              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
+              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
+              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
+              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
+            }
+          }
+        }
+        float4* dst = P.group_partial + (long long)gi * 64 + 2 * lane;
+        dst[0] = lo;
+        dst[1] = hi;
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          red_add_release(P.unit_counter + u, 1);
+        }
+        gi += P.grid;
+      } else {
+        const float4* src = P.group_partial + (long long)un * P.NG * 64 + 2 * lane;
+#pragma unroll 2
+        for (int r = 0; r < P.NG; ++r) {
+          const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
+          combine(lo.x, lo.y, v0.x, v0.y);
+          combine(lo.z, lo.w, v0.z, v0.w);
+          combine(hi.x, hi.y, v1.x, v1.y);
+          combine(hi.z, hi.w, v1.z, v1.w);
+        }
+        unsigned int* out = P.lse2 + (long long)un * kRows + 4 * lane;
+        st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
+        st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
+        st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
+        st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
+        un += P.grid;
+      }
     }
   }
 

@@ -167,3 +167,33 @@ def test_unstructured_variant(Hkv, frac, order):
         kvc.kvc_gather_unstructured(desc, wl.k, wl.v, idx2, n2, o2, B, k2, v2)
         assert torch.equal(k2.view(torch.uint8), k_out.view(torch.uint8)) and torch.equal(v2.view(torch.uint8), v_out.view(torch.uint8))
     assert torch.equal(n2, n_keep) and torch.equal(o2, off)
+    # the fused entry without the optional outputs (the sorted scores then take the place of the scores in
+    # the workspace) gives the same compressed cache
+    k3 = torch.empty_like(k_out); v3 = torch.empty_like(v_out)
+    n3 = torch.empty_like(n_keep); o3 = torch.empty_like(off)
+    kvc.kvc_compress_unstructured(desc, wl.q, wl.k, wl.v, B, k3, v3, n3, o3, None, None, status, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(n3, n_keep) and torch.equal(o3, off)
+    assert torch.equal(k3.view(torch.uint8), k_out.view(torch.uint8)) and torch.equal(v3.view(torch.uint8), v_out.view(torch.uint8))
+
+
+def test_unstructured_variant_with_value_norm_weighting():
+    """The two variants together: weighted scores feed the per-head selection."""
+    import oracle
+    cfg = W.WorkloadConfig("unstructured_vnorm", 2, 8, 2, 128, 700, 32, batch=1, dtype="bf16", elem_std=1.0)
+    dev, wl, desc = _setup(cfg, value_norm=1)
+    L, Hkv, N, d = cfg.n_layers, cfg.n_kv_heads, cfg.n_ctx, cfg.head_dim
+    B = int(0.2 * L * Hkv * N)
+    ws = torch.empty(kvc.kvc_workspace_size(desc, 0), dtype=torch.uint8, device=dev)
+    k_out = torch.empty((1, B * d), dtype=wl.k[0].dtype, device=dev); v_out = torch.empty_like(k_out)
+    n_keep = torch.empty((1, L, Hkv), dtype=torch.int32, device=dev)
+    off = torch.empty((1, L * Hkv + 1), dtype=torch.int64, device=dev)
+    scores = torch.empty((L, 1, Hkv, N), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    kvc.kvc_compress_unstructured(desc, wl.q, wl.k, wl.v, B, k_out, v_out, n_keep, off, None, scores, status, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    S = _host(scores)
+    Pz.assert_scores_close(S, _oracle_vnorm_scores(wl, desc))
+    n_ref, off_ref = oracle.select_unstructured(S[:, 0].astype(np.float64), B)
+    assert np.array_equal(n_ref, _host(n_keep)[0]) and np.array_equal(off_ref, _host(off)[0])
