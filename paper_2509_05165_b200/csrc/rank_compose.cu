@@ -2,16 +2,24 @@
 //
 // Every (layer, sequence, KV head) is one segment of N (score, position) pairs that must come
 // out in descending score order with equal scores in ascending position.  Scores are mapped to
-// 32-bit keys whose ascending order is the wanted order, and all segments are sorted together by
-// a stable least-significant-digit radix sort (8-bit digits, 4 passes) over tiles of 4096
-// elements.  A pass is two kernels: one counts the digit of every tile, the other gives every
-// tile its own CTA, which derives the tile's output ranges from the counts of its segment,
-// ranks its elements, reorders them by digit in shared memory and writes them out in runs.
-// Tiles are independent inside a pass, so the whole GPU is busy whatever the number of
-// segments; the passes ping-pong between two scratch buffers that stay in L2.  The last pass
-// writes the positions straight into idx and leaves the sorted keys for the composite kernel,
-// which turns them back into scores and reduces over the heads.
+// 32-bit keys whose ascending order is the wanted order; the sort is a stable least-significant-
+// digit radix sort, in one of two forms:
+//
+//   N <= 32768   one CTA per segment, the whole sort inside one SM's shared memory (4-bit digits,
+//                thread-private counters, the permutation updated in place); one launch.
+//   larger N     all segments together over tiles of 4096 elements (8-bit digits, 4 passes).  A
+//                pass is two kernels: one counts the digit of every tile, the other gives every
+//                tile its own CTA, which derives the tile's output ranges from the counts of its
+//                segment, ranks its elements, reorders them by digit in shared memory and writes
+//                them out in runs.  Tiles are independent inside a pass, so the whole GPU is busy
+//                whatever the number of segments; the passes ping-pong between two scratch
+//                buffers that stay in L2.
+//
+// Either way the positions go straight into idx and the sorted keys are left for the composite
+// kernel, which turns them back into scores and reduces over the heads.
 #include "kvc_internal.cuh"
+
+#include <mutex>
 
 namespace kvc {
 namespace {
@@ -222,6 +230,287 @@ sort_scatter_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Segments of at most kSegMaxN elements: one CTA sorts one whole segment inside its SM.
+//
+// A stable least-significant-digit sort with 4-bit digits.  The keys are read from global memory
+// once and stay in shared memory, by position; what moves between the passes is a permutation of
+// 16-bit positions, in place.  Thread t owns the places [t * ipt, (t + 1) * ipt) of the current
+// order.  A pass:
+//   count    every thread walks its places in order: position -> byte of the key -> digit, and a
+//            counter of its own per digit (shared memory, one bank per lane): the value it finds
+//            is the element's rank among the thread's elements of that digit.  No work crosses
+//            lanes, so nothing depends on how the digits are distributed.
+//   scan     exclusive prefix over (digit, thread), digits ascending: the first place of every
+//            thread's elements of every digit.
+//   scatter  position -> place = first place + rank.  Every thread read all of its places
+//            before the scan, so the permutation is overwritten in place.
+// (thread, place inside the thread) is the order itself, so every pass is stable, and with the
+// identity as the first order equal keys stay in ascending position.  A digit that all keys of
+// the segment share orders nothing and its pass is left out (scores in [2^-31, 2) share the
+// top one).  After the last pass positions and keys go out through the permutation, coalesced.
+// Global traffic: scores read once, idx and sorted keys written once; one launch.
+constexpr int kSegMaxN = 32768;
+constexpr int kSegMaxIpt = 32;                 // places per thread
+constexpr int kSegBatch = 4;                   // key lookups in flight per thread
+constexpr int kMaxDevices = 64;
+
+__device__ __forceinline__ uint32_t lds_u8(uint32_t a) { uint32_t v; asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v; }
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) { uint32_t v; asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v; }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) { uint32_t v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v; }
+__device__ __forceinline__ uint4 lds_v4(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t a, uint32_t v) { asm volatile("st.shared.u16 [%0], %1;" :: "r"(a), "h"((unsigned short)v) : "memory"); }
+__device__ __forceinline__ void sts_u32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" :: "r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void sts_v4(uint32_t a, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Shared-memory map of a segment of N elements sorted by T threads (byte offsets).
+struct SegLayout {
+  int n_pad;            // N rounded up to 32: key_slot and place_slot permute inside aligned blocks of 32
+  int lg;               // log2 of the places per thread
+  uint32_t keys;        // uint32[n_pad]: the keys, by position
+  uint32_t perm;        // uint16[n_pad]: the position at every place
+  uint32_t cnt;         // uint16[8][T][2]: thread t's counter of digit d in row d & 7, half d >> 3
+  uint32_t wtot;        // uint32[32]: the scan's warp totals;  uint32: bits that differ between keys
+  uint32_t total;
+};
+__host__ __device__ inline SegLayout seg_layout(long long N, int T) {
+  SegLayout s;
+  s.n_pad = (int)((N + 31) / 32 * 32);
+  s.lg = 0;
+  while (((long long)T << s.lg) < N) ++s.lg;
+  s.keys = 0;
+  s.perm = 4u * s.n_pad;
+  s.cnt = s.perm + 2u * s.n_pad;
+  s.wtot = s.cnt + 8u * T * 4u;
+  s.total = s.wtot + 256u;
+  return s;
+}
+
+// Where things sit, to keep the banks apart.  Key of position i: word i ^ ((i >> 5) & 31): the
+// threads of a warp start 32 places apart, which in the first pass are 32 positions apart.
+// Place j: halfword j ^ (((j >> 6) & 3) << 3): a warp reads 32 stretches of 64 bytes, 16 at a time.
+__device__ __forceinline__ uint32_t key_slot(uint32_t i) { return i ^ ((i >> 5) & 31u); }
+__device__ __forceinline__ uint32_t place_slot(uint32_t j) { return j ^ (((j >> 6) & 3u) << 3); }
+
+// score_to_key without the branch.
+__device__ __forceinline__ uint32_t seg_key(float f) {
+  uint32_t b = __float_as_uint(f);
+  b = (b == 0x80000000u) ? 0u : b;
+  const uint32_t m = (uint32_t)((int32_t)b >> 31) | 0x80000000u;
+  return ~(b ^ m);
+}
+
+// Every group of 4 consecutive keys of the segment goes to use(i, k0, k1, k2, k3, n): i = position
+// of the first (a multiple of 4), n = how many of the 4 exist.  With 16-byte aligned scores all of
+// a thread's loads are issued before the first use.
+template <int T, typename F>
+__device__ __forceinline__ void seg_for_keys(const float* s_in, int N, int tid, F use) {
+  constexpr int kGroups = kSegMaxIpt / 4;
+  const bool wide = (reinterpret_cast<uintptr_t>(s_in) & 15u) == 0 && N >= 4;
+  if (wide) {
+    const int last = (N & ~3) - 4;                           // first position of the last whole group
+    float4 v[kGroups];
+#pragma unroll
+    for (int g = 0; g < kGroups; ++g) v[g] = *reinterpret_cast<const float4*>(s_in + min((g * T + tid) * 4, last));
+#pragma unroll
+    for (int g = 0; g < kGroups; ++g) {
+      const int i = (g * T + tid) * 4;
+      if (i + 4 <= N) use(i, seg_key(v[g].x), seg_key(v[g].y), seg_key(v[g].z), seg_key(v[g].w), 4);
+    }
+    if (tid == 0 && (N & 3)) {
+      const int i = N & ~3;
+      use(i, seg_key(s_in[i]), seg_key(i + 1 < N ? s_in[i + 1] : 0.f), seg_key(i + 2 < N ? s_in[i + 2] : 0.f), seg_key(0.f), N - i);
+    }
+  } else {
+    for (int i = tid * 4; i < N; i += T * 4)
+      use(i, seg_key(s_in[i]), seg_key(i + 1 < N ? s_in[i + 1] : 0.f), seg_key(i + 2 < N ? s_in[i + 2] : 0.f),
+          seg_key(i + 3 < N ? s_in[i + 3] : 0.f), min(4, N - i));
+  }
+}
+
+template <int T>
+__global__ void __launch_bounds__(T, T == 1024 ? 1 : 4)
+segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ keys_out,
+                    int32_t* __restrict__ idx_out, int N) {
+  constexpr int kRowShift = (T == 1024) ? 12 : 10;          // log2 of a row of counters in bytes
+  static_assert(T == 1024 || T == 256, "row shift");
+  constexpr int kScanWarps = T / 64;                        // the scan runs on the first T / 2 threads
+  extern __shared__ __align__(16) unsigned char seg_smem[];
+  const SegLayout lay = seg_layout(N, T);
+  const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(seg_smem);
+  const uint32_t keys = sbase + lay.keys, perm = sbase + lay.perm, cnt = sbase + lay.cnt, wtot = sbase + lay.wtot;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lg = lay.lg, ipt = 1 << lg;
+  const int j0 = tid << lg;
+  const int nv = max(0, min(ipt, N - j0));                   // my places: j0 .. j0 + nv - 1
+  // My counter of digit d: + ((d & 7) << kRowShift) + ((d >> 3) << 1).  Inside a warp's 32 columns, groups
+  // of 4 are permuted by the warp number so that the scan's 16-byte reads of neighbouring columns spread
+  // over the banks; a lane keeps a bank of its own.
+  const uint32_t cbase = cnt + (uint32_t)(tid ^ (((tid >> 5) & 3) << 2)) * 4u;
+
+  grid_dependency_wait();
+  const float* s_in = scores + (long long)blockIdx.x * N;
+
+  // ---- the keys, once; the identity as the first order; which bits differ anywhere in the segment
+  uint32_t diff = 0;
+  {
+    const uint32_t ref = seg_key(s_in[0]);
+    if (tid == 0) sts_u32(wtot + 128, 0u);
+    seg_for_keys<T>(s_in, N, tid, [&](int i, uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3, int n) {
+      const uint32_t sw = ((uint32_t)i >> 5) & 31u;          // the four stay inside their 16 bytes; the table is padded
+      sts_u32(keys + (((uint32_t)i) ^ sw) * 4u, k0);
+      sts_u32(keys + (((uint32_t)i + 1u) ^ sw) * 4u, k1);
+      sts_u32(keys + (((uint32_t)i + 2u) ^ sw) * 4u, k2);
+      sts_u32(keys + (((uint32_t)i + 3u) ^ sw) * 4u, k3);
+      diff |= k0 ^ ref;
+      if (n > 1) diff |= k1 ^ ref;
+      if (n > 2) diff |= k2 ^ ref;
+      if (n > 3) diff |= k3 ^ ref;
+    });
+    if (lg >= 3) {
+#pragma unroll
+      for (int q = 0; q < kSegMaxIpt / 8; ++q) {
+        if (q * 8 < nv) {
+          const uint32_t j = (uint32_t)(j0 + q * 8), jj = j * 0x10001u;         // j in both halves
+          sts_v4(perm + place_slot(j) * 2u, make_uint4(jj + 0x10000u, jj + 0x30002u, jj + 0x50004u, jj + 0x70006u));
+        }
+      }
+    } else {
+      for (int k = 0; k < nv; ++k) sts_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u, (uint32_t)(j0 + k));
+    }
+    diff = __reduce_or_sync(0xffffffffu, diff);
+    __syncthreads();
+    if (lane == 0 && diff != 0) atomicOr(reinterpret_cast<uint32_t*>(seg_smem + lay.wtot + 128), diff);
+    __syncthreads();
+    diff = lds_u32(wtot + 128);
+  }
+
+#pragma unroll 1
+  for (int B = 0; B < 4; ++B) {
+    const uint32_t kb = keys + (uint32_t)B;                  // byte B of the key of position i: kb + 4 key_slot(i)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (((diff >> (8 * B + 4 * h)) & 15u) == 0) continue;  // a digit every key shares orders nothing
+      // with an element as  position | byte << 16 | rank << 24,  its digit d sits at bit 16 + 4 h
+      constexpr uint32_t kRowMask = 7u << kRowShift;
+      const int sh_row = 16 + 4 * h - kRowShift, sh_half = 18 + 4 * h;
+
+      // ---- count
+#pragma unroll
+      for (int d = 0; d < 8; ++d) sts_u32(cbase + ((uint32_t)d << kRowShift), 0u);
+      uint32_t packed[kSegMaxIpt];
+      if (lg >= 3) {
+#pragma unroll
+        for (int q = 0; q < kSegMaxIpt / 8; ++q) {
+          if (q * 8 < nv) {
+            const uint4 w = lds_v4(perm + place_slot((uint32_t)(j0 + q * 8)) * 2u);
+            packed[q * 8 + 0] = w.x & 0xffffu; packed[q * 8 + 1] = w.x >> 16;
+            packed[q * 8 + 2] = w.y & 0xffffu; packed[q * 8 + 3] = w.y >> 16;
+            packed[q * 8 + 4] = w.z & 0xffffu; packed[q * 8 + 5] = w.z >> 16;
+            packed[q * 8 + 6] = w.w & 0xffffu; packed[q * 8 + 7] = w.w >> 16;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) if (k < nv) packed[k] = lds_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u);
+      }
+#pragma unroll
+      for (int k0 = 0; k0 < kSegMaxIpt; k0 += kSegBatch) {
+        uint32_t b[kSegBatch];
+#pragma unroll
+        for (int k = 0; k < kSegBatch; ++k) if (k0 + k < nv) b[k] = lds_u8(kb + key_slot(packed[k0 + k]) * 4u);
+#pragma unroll
+        for (int k = 0; k < kSegBatch; ++k) {
+          if (k0 + k < nv) {
+            const uint32_t pk = packed[k0 + k] | (b[k] << 16);
+            const uint32_t a = cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u));
+            const uint32_t seen = lds_u16(a);
+            sts_u16(a, seen + 1u);
+            packed[k0 + k] = pk + (seen << 24);
+          }
+        }
+      }
+      __syncthreads();
+
+      // ---- scan.  Thread s < T / 2 owns 16 neighbouring threads' counters of the digits in its row: the low
+      //      halves (digit = row) precede all high halves (digit = row + 8) in the order of the places.
+      {
+        const uint32_t mine = cnt + (uint32_t)tid * 64u;
+        const uint32_t rot = (((uint32_t)tid >> 1) & 3u) << 4;                     // the permutation of cbase, seen from here
+        uint32_t lo_sum = 0, hi_sum = 0, lo_incl = 0, hi_incl = 0;
+        if (tid < T / 2) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 w = lds_v4(mine + ((q * 16) ^ rot));
+            lo_sum += (w.x & 0xffffu) + (w.y & 0xffffu) + (w.z & 0xffffu) + (w.w & 0xffffu);
+            hi_sum += (w.x >> 16) + (w.y >> 16) + (w.z >> 16) + (w.w >> 16);
+          }
+          lo_incl = lo_sum; hi_incl = hi_sum;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t x = __shfl_up_sync(0xffffffffu, lo_incl, o);
+            const uint32_t y = __shfl_up_sync(0xffffffffu, hi_incl, o);
+            if (lane >= o) { lo_incl += x; hi_incl += y; }
+          }
+          if (lane == 31) { sts_u32(wtot + warp * 4, lo_incl); sts_u32(wtot + (kScanWarps + warp) * 4, hi_incl); }
+        }
+        __syncthreads();
+        if (tid < T / 2) {
+          const uint32_t x = lane < 2 * kScanWarps ? lds_u32(wtot + lane * 4) : 0u;
+          uint32_t e = x;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, e, o);
+            if (lane >= o) e += y;
+          }
+          e -= x;                                                                  // exclusive over the warp totals
+          uint32_t lo = __shfl_sync(0xffffffffu, e, warp) + lo_incl - lo_sum;
+          uint32_t hi = __shfl_sync(0xffffffffu, e, kScanWarps + warp) + hi_incl - hi_sum;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t a = mine + ((q * 16) ^ rot);
+            const uint4 w = lds_v4(a);
+            uint4 o4;
+            o4.x = lo | (hi << 16); lo += w.x & 0xffffu; hi += w.x >> 16;
+            o4.y = lo | (hi << 16); lo += w.y & 0xffffu; hi += w.y >> 16;
+            o4.z = lo | (hi << 16); lo += w.z & 0xffffu; hi += w.z >> 16;
+            o4.w = lo | (hi << 16); lo += w.w & 0xffffu; hi += w.w >> 16;
+            sts_v4(a, o4);
+          }
+        }
+      }
+      __syncthreads();
+
+      // ---- scatter (in place: every place was read before the scan)
+#pragma unroll
+      for (int k = 0; k < kSegMaxIpt; ++k) {
+        if (k < nv) {
+          const uint32_t pk = packed[k];
+          const uint32_t off = lds_u16(cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u)));
+          sts_u16(perm + place_slot(off + (pk >> 24)) * 2u, pk);
+        }
+      }
+      __syncthreads();
+    }
+  }
+
+  // ---- out: the positions, and the keys through them
+  uint32_t* k_out = keys_out + (long long)blockIdx.x * N;
+  int32_t* i_out = idx_out + (long long)blockIdx.x * N;
+  for (int j = tid; j < N; j += T) {
+    const uint32_t q = lds_u16(perm + place_slot((uint32_t)j) * 2u);
+    i_out[j] = (int32_t)q;
+    k_out[j] = lds_u32(keys + key_slot(q) * 4u);
+  }
+}
+
 // Eq. 19 over the sorted keys: composite[lb, k] = agg_head_h score(keys[lb, h, k]).
 // Mean: heads added in ascending order in fp32, one division at the end.
 __global__ void compose_kernel(const uint32_t* __restrict__ keys, float* __restrict__ composite,
@@ -248,6 +537,30 @@ __global__ void sorted_scores_kernel(const uint32_t* __restrict__ keys, float* _
 }
 
 }  // namespace
+
+// Can a segment of N elements be sorted inside one SM here?  Sets the shared-memory attribute once
+// per device (it is per device), under a lock.  *threads = the CTA size to launch.
+static kvc_status segment_sort_prepare(long long N, int* threads) {
+  if (N > kSegMaxN) return KVC_ERR_UNSUPPORTED;
+  static std::mutex mu;
+  static int optin[kMaxDevices];           // 0: not looked at, else the device's opt-in bytes (or -1)
+  int dev = 0;
+  KVC_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return KVC_ERR_UNSUPPORTED;
+  const int T = N > 8192 ? 1024 : 256;
+  const size_t need = seg_layout(N, T).total;
+  std::lock_guard<std::mutex> lock(mu);
+  if (optin[dev] == 0) {
+    int bytes = 0;
+    KVC_CUDA(cudaDeviceGetAttribute(&bytes, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    KVC_CUDA(cudaFuncSetAttribute(segment_sort_kernel<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    KVC_CUDA(cudaFuncSetAttribute(segment_sort_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    optin[dev] = bytes > 0 ? bytes : -1;
+  }
+  if (optin[dev] < 0 || need > (size_t)optin[dev]) return KVC_ERR_UNSUPPORTED;
+  *threads = T;
+  return KVC_OK;
+}
 
 static int sort_tiles(const Problem& P) { return (int)((P.N + kTileItems - 1) / kTileItems); }
 
@@ -282,13 +595,31 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
   buf.vals_b = reinterpret_cast<int32_t*>(w + 3 * region);
   uint32_t* counts = reinterpret_cast<uint32_t*>(w + 4 * region);
   const long long segments = (long long)P.L * P.Bt * P.Hkv;
+  int seg_threads = 0;
+  const kvc_status seg_state = segment_sort_prepare(P.N, &seg_threads);
+  if (seg_state != KVC_OK && seg_state != KVC_ERR_UNSUPPORTED) return seg_state;
   const int tiles = sort_tiles(P);
   const long long blocks = segments * tiles;
-  if (blocks >= (1LL << 31)) {
+  if (seg_state == KVC_OK) {
+    // a segment fits one SM's shared memory: the whole sort in one launch, one CTA per segment
+    if (segments >= (1LL << 31)) {
+      set_error("compose: too many segments");
+      return KVC_ERR_UNSUPPORTED;
+    }
+    const size_t smem = seg_layout(P.N, seg_threads).total;
+    if (seg_threads == 1024) {
+      KVC_CUDA(launch_dependent(segment_sort_kernel<1024>, dim3((unsigned)segments), dim3(1024), smem, st,
+                                scores, buf.keys_b, idx, (int)P.N));
+    } else {
+      KVC_CUDA(launch_dependent(segment_sort_kernel<256>, dim3((unsigned)segments), dim3(256), smem, st,
+                                scores, buf.keys_b, idx, (int)P.N));
+    }
+    KVC_LAUNCH_CHECK("segment_sort_kernel");
+  } else if (blocks >= (1LL << 31)) {
     set_error("compose: too many sort tiles");
     return KVC_ERR_UNSUPPORTED;
   }
-  for (int pass = 0; pass < 4; ++pass) {
+  for (int pass = 0; pass < 4 && seg_state != KVC_OK; ++pass) {
     KVC_CUDA(launch_dependent(sort_count_kernel, dim3((unsigned)blocks), dim3(kSortThreads), 0, st,
                               scores, buf, idx, counts, P.N, tiles, pass));
     KVC_LAUNCH_CHECK("sort_count_kernel");

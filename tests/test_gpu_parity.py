@@ -340,6 +340,36 @@ def test_exact_ties_are_broken_by_position_and_layer():
     assert off.cpu().tolist() == [[0, 900, 990, 1000, 1000]]
 
 
+@pytest.mark.parametrize("N", [1, 2, 31, 33, 255, 257, 400, 1000, 4095, 4097, 8191, 8192, 8193, 12345,
+                               32767, 32768, 32769, 40000])
+def test_ranking_alone_across_lengths_and_both_sorts(N):
+    """Eqs. 17-19 on scores given by the caller: lengths on both sides of every switch of the
+    ranking (places per thread, CTA size, one SM per segment or all segments over tiles), segments
+    that do not start on 16 bytes, and values of every kind -- long runs of equal scores, both
+    zeros, negatives, denormals, huge values."""
+    dev = _cuda()
+    L, Hkv = 2, 3
+    cfg = W.WorkloadConfig("rank", L, Hkv, Hkv, 64, N, 1, dtype="f32", elem_std=1.0)
+    desc = kvc.desc_from_config(cfg)
+    g = np.random.default_rng(1234 + N)
+    S = np.empty((L, 1, Hkv, N), dtype=np.float32)
+    S[0, 0, 0] = g.random(N, dtype=np.float32) / max(N, 1)                  # probabilities, one exponent range
+    S[0, 0, 1] = np.round(g.random(N) * 7).astype(np.float32) / 7           # eight values: long ties
+    S[0, 0, 2] = np.exp(g.normal(0, 12, N)).astype(np.float32)              # forty orders of magnitude
+    S[1, 0, 0] = g.normal(0, 1, N).astype(np.float32)                       # both signs
+    S[1, 0, 1] = 0.25                                                       # all equal: no pass orders anything
+    special = np.array([0.0, -0.0, 1e-45, -1e-45, 1.0, -1.0, 3e38, -3e38, 1e-38, 2.0 ** -31], dtype=np.float32)
+    S[1, 0, 2] = special[g.integers(0, len(special), N)]
+    scores = torch.from_numpy(S).to(dev)
+    idx = torch.empty((L, 1, Hkv, N), dtype=torch.int32, device=dev)
+    comp = torch.empty((L, 1, N), dtype=torch.float32, device=dev)
+    ws = torch.empty(kvc.kvc_workspace_size(desc, 0), dtype=torch.uint8, device=dev)
+    kvc.kvc_compose(desc, scores, idx, comp, ws)
+    torch.cuda.synchronize()
+    Pz.assert_rank_exact(S, _host(idx))
+    Pz.assert_compose_exact(S, _host(idx), _host(comp), desc.agg_head)
+
+
 def test_argument_errors_are_reported_not_launched():
     dev = _cuda()
     cfg = W.WorkloadConfig("err", 1, 2, 1, 64, 64, 4, dtype="f32", elem_std=1.0)
