@@ -20,6 +20,7 @@
 #include "kvc_internal.cuh"
 
 #include <mutex>
+#include <type_traits>
 
 namespace kvc {
 namespace {
@@ -274,7 +275,7 @@ struct SegLayout {
   int n_pad;            // N rounded up to 32: key_slot and place_slot permute inside aligned blocks of 32
   int lg;               // log2 of the places per thread
   uint32_t keys;        // uint32[n_pad]: the keys, by position
-  uint32_t perm;        // uint16[n_pad]: the position at every place
+  uint32_t perm;        // uint16[n_pad]: the key slot (key_slot of the position) at every place
   uint32_t cnt;         // uint16[8][T][2]: thread t's counter of digit d in row d & 7, half d >> 3
   uint32_t wtot;        // uint32[32]: the scan's warp totals;  uint32: bits that differ between keys
   uint32_t total;
@@ -350,6 +351,7 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
   const int lg = lay.lg, ipt = 1 << lg;
   const int j0 = tid << lg;
   const int nv = max(0, min(ipt, N - j0));                   // my places: j0 .. j0 + nv - 1
+  const bool full = __all_sync(0xffffffffu, nv == kSegMaxIpt);   // the warp's decision
   // My counter of digit d: + ((d & 7) << kRowShift) + ((d >> 3) << 1).  Inside a warp's 32 columns, groups
   // of 4 are permuted by the warp number so that the scan's 16-byte reads of neighbouring columns spread
   // over the banks; a lane keeps a bank of its own.
@@ -374,16 +376,21 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
       if (n > 2) diff |= k2 ^ ref;
       if (n > 3) diff |= k3 ^ ref;
     });
+    // (the permutation holds key slots, not positions: a lookup needs no translation)
     if (lg >= 3) {
 #pragma unroll
       for (int q = 0; q < kSegMaxIpt / 8; ++q) {
         if (q * 8 < nv) {
-          const uint32_t j = (uint32_t)(j0 + q * 8), jj = j * 0x10001u;         // j in both halves
-          sts_v4(perm + place_slot(j) * 2u, make_uint4(jj + 0x10000u, jj + 0x30002u, jj + 0x50004u, jj + 0x70006u));
+          const uint32_t j = (uint32_t)(j0 + q * 8);
+          // j is a multiple of 8: the eight slots are (j ^ m's high bits) | (e ^ m's low 3 bits), e = 0..7
+          const uint32_t m = (j >> 5) & 31u;
+          const uint32_t bb = (j ^ (m & 24u)) * 0x10001u, mm = (m & 7u) * 0x10001u;
+          sts_v4(perm + place_slot(j) * 2u, make_uint4(bb | (0x10000u ^ mm), bb | (0x30002u ^ mm),
+                                                         bb | (0x50004u ^ mm), bb | (0x70006u ^ mm)));
         }
       }
     } else {
-      for (int k = 0; k < nv; ++k) sts_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u, (uint32_t)(j0 + k));
+      for (int k = 0; k < nv; ++k) sts_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u, key_slot((uint32_t)(j0 + k)));
     }
     diff = __reduce_or_sync(0xffffffffu, diff);
     __syncthreads();
@@ -394,49 +401,53 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
 
 #pragma unroll 1
   for (int B = 0; B < 4; ++B) {
-    const uint32_t kb = keys + (uint32_t)B;                  // byte B of the key of position i: kb + 4 key_slot(i)
+    const uint32_t kb = keys + (uint32_t)B;                  // byte B of the key in slot s: kb + 4 s
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       if (((diff >> (8 * B + 4 * h)) & 15u) == 0) continue;  // a digit every key shares orders nothing
-      // with an element as  position | byte << 16 | rank << 24,  its digit d sits at bit 16 + 4 h
+      // with an element as  key slot | byte << 16 | rank << 24,  its digit d sits at bit 16 + 4 h
       constexpr uint32_t kRowMask = 7u << kRowShift;
       const int sh_row = 16 + 4 * h - kRowShift, sh_half = 18 + 4 * h;
 
-      // ---- count
+      // ---- count (threads whose 32 places all exist take the copy without the per-place tests)
 #pragma unroll
       for (int d = 0; d < 8; ++d) sts_u32(cbase + ((uint32_t)d << kRowShift), 0u);
       uint32_t packed[kSegMaxIpt];
-      if (lg >= 3) {
+      auto count = [&](auto full_tag) {
+        constexpr bool kFull = decltype(full_tag)::value;
+        if (kFull || lg >= 3) {
 #pragma unroll
-        for (int q = 0; q < kSegMaxIpt / 8; ++q) {
-          if (q * 8 < nv) {
-            const uint4 w = lds_v4(perm + place_slot((uint32_t)(j0 + q * 8)) * 2u);
-            packed[q * 8 + 0] = w.x & 0xffffu; packed[q * 8 + 1] = w.x >> 16;
-            packed[q * 8 + 2] = w.y & 0xffffu; packed[q * 8 + 3] = w.y >> 16;
-            packed[q * 8 + 4] = w.z & 0xffffu; packed[q * 8 + 5] = w.z >> 16;
-            packed[q * 8 + 6] = w.w & 0xffffu; packed[q * 8 + 7] = w.w >> 16;
+          for (int q = 0; q < kSegMaxIpt / 8; ++q) {
+            if (kFull || q * 8 < nv) {
+              const uint4 w = lds_v4(perm + place_slot((uint32_t)(j0 + q * 8)) * 2u);
+              packed[q * 8 + 0] = w.x & 0xffffu; packed[q * 8 + 1] = w.x >> 16;
+              packed[q * 8 + 2] = w.y & 0xffffu; packed[q * 8 + 3] = w.y >> 16;
+              packed[q * 8 + 4] = w.z & 0xffffu; packed[q * 8 + 5] = w.z >> 16;
+              packed[q * 8 + 6] = w.w & 0xffffu; packed[q * 8 + 7] = w.w >> 16;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) if (k < nv) packed[k] = lds_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u);
+        }
+#pragma unroll
+        for (int k0 = 0; k0 < kSegMaxIpt; k0 += kSegBatch) {
+          uint32_t b[kSegBatch];
+#pragma unroll
+          for (int k = 0; k < kSegBatch; ++k) if (kFull || k0 + k < nv) b[k] = lds_u8(kb + packed[k0 + k] * 4u);
+#pragma unroll
+          for (int k = 0; k < kSegBatch; ++k) {
+            if (kFull || k0 + k < nv) {
+              const uint32_t pk = packed[k0 + k] | (b[k] << 16);
+              const uint32_t a = cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u));
+              const uint32_t seen = lds_u16(a);
+              sts_u16(a, seen + 1u);
+              packed[k0 + k] = pk + (seen << 24);
+            }
           }
         }
-      } else {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) if (k < nv) packed[k] = lds_u16(perm + place_slot((uint32_t)(j0 + k)) * 2u);
-      }
-#pragma unroll
-      for (int k0 = 0; k0 < kSegMaxIpt; k0 += kSegBatch) {
-        uint32_t b[kSegBatch];
-#pragma unroll
-        for (int k = 0; k < kSegBatch; ++k) if (k0 + k < nv) b[k] = lds_u8(kb + key_slot(packed[k0 + k]) * 4u);
-#pragma unroll
-        for (int k = 0; k < kSegBatch; ++k) {
-          if (k0 + k < nv) {
-            const uint32_t pk = packed[k0 + k] | (b[k] << 16);
-            const uint32_t a = cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u));
-            const uint32_t seen = lds_u16(a);
-            sts_u16(a, seen + 1u);
-            packed[k0 + k] = pk + (seen << 24);
-          }
-        }
-      }
+      };
+      if (full) count(std::true_type{}); else count(std::false_type{});
       __syncthreads();
 
       // ---- scan.  Thread s < T / 2 owns 16 neighbouring threads' counters of the digits in its row: the low
@@ -489,25 +500,29 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
       __syncthreads();
 
       // ---- scatter (in place: every place was read before the scan)
+      auto scatter = [&](auto full_tag) {
+        constexpr bool kFull = decltype(full_tag)::value;
 #pragma unroll
-      for (int k = 0; k < kSegMaxIpt; ++k) {
-        if (k < nv) {
-          const uint32_t pk = packed[k];
-          const uint32_t off = lds_u16(cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u)));
-          sts_u16(perm + place_slot(off + (pk >> 24)) * 2u, pk);
+        for (int k = 0; k < kSegMaxIpt; ++k) {
+          if (kFull || k < nv) {
+            const uint32_t pk = packed[k];
+            const uint32_t off = lds_u16(cbase + (((pk >> sh_row) & kRowMask) | ((pk >> sh_half) & 2u)));
+            sts_u16(perm + place_slot(off + (pk >> 24)) * 2u, pk);
+          }
         }
-      }
+      };
+      if (full) scatter(std::true_type{}); else scatter(std::false_type{});
       __syncthreads();
     }
   }
 
-  // ---- out: the positions, and the keys through them
+  // ---- out: the positions (a slot's position is key_slot of it: the map is its own inverse), and the keys
   uint32_t* k_out = keys_out + (long long)blockIdx.x * N;
   int32_t* i_out = idx_out + (long long)blockIdx.x * N;
   for (int j = tid; j < N; j += T) {
     const uint32_t q = lds_u16(perm + place_slot((uint32_t)j) * 2u);
-    i_out[j] = (int32_t)q;
-    k_out[j] = lds_u32(keys + key_slot(q) * 4u);
+    i_out[j] = (int32_t)key_slot(q);
+    k_out[j] = lds_u32(keys + q * 4u);
   }
 }
 
