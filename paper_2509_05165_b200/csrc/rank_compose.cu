@@ -2,21 +2,13 @@
 //
 // Every (layer, sequence, KV head) is one segment of N (score, position) pairs that must come
 // out in descending score order with equal scores in ascending position.  Scores are mapped to
-// 32-bit keys whose ascending order is the wanted order; the sort is a stable least-significant-
-// digit radix sort, in one of two forms:
+// 32-bit keys whose ascending order is the wanted order.  A segment of up to 32768 elements is
+// sorted by one CTA inside its SM's shared memory (a stable least-significant-digit radix sort
+// with 4-bit digits, thread-private counters, the permutation updated in place): one launch.  A
+// longer segment is cut into such chunks, which are then merged pairwise (merge path), one launch
+// per level.
 //
-//   N <= 32768   one CTA per segment, the whole sort inside one SM's shared memory (4-bit digits,
-//                thread-private counters, the permutation updated in place); one launch.
-//   larger N     all segments together over tiles of 4096 elements (8-bit digits, 4 passes).  A
-//                pass is two kernels: one counts the digit of every tile, the other gives every
-//                tile its own CTA, which derives the tile's output ranges from the counts of its
-//                segment, ranks its elements, reorders them by digit in shared memory and writes
-//                them out in runs.  Tiles are independent inside a pass, so the whole GPU is busy
-//                whatever the number of segments; the passes ping-pong between two scratch
-//                buffers that stay in L2.
-//
-// Either way the positions go straight into idx and the sorted keys are left for the composite
-// kernel, which turns them back into scores and reduces over the heads.
+// The positions go straight into idx and the sorted keys are left for the composite kernel, which turns them back into scores and reduces over the heads.
 #include "kvc_internal.cuh"
 
 #include <mutex>
@@ -24,212 +16,6 @@
 
 namespace kvc {
 namespace {
-
-constexpr int kSortThreads = 512;
-constexpr int kWarps = kSortThreads / 32;
-constexpr int kRadix = 256;
-constexpr int kItems = 8;                               // elements per thread
-constexpr int kTileItems = kSortThreads * kItems;       // 4096 elements per tile
-constexpr int kWarpItems = 32 * kItems;                 // a warp owns 256 consecutive elements of a tile
-
-struct SortBuffers {
-  uint32_t* keys_a; int32_t* vals_a;
-  uint32_t* keys_b; int32_t* vals_b;
-};
-
-// Lanes of the warp whose 8-bit digit equals this lane's (0 for a lane without an element).
-// Eight ballots: the cost does not depend on how many different digits the warp holds.
-__device__ __forceinline__ uint32_t same_digit_lanes(uint32_t digit, bool valid) {
-  uint32_t peers = __ballot_sync(0xffffffffu, valid);
-#pragma unroll
-  for (int b = 0; b < 8; ++b) {
-    const bool bit = (digit >> b) & 1u;
-    const uint32_t m = __ballot_sync(0xffffffffu, bit);
-    peers &= bit ? m : ~m;
-  }
-  return valid ? peers : 0u;
-}
-
-// Source and destination of a pass.  0: scores -> A;  1: A -> B;  2: B -> A;  3: A -> (keys_b, idx).
-struct PassIo {
-  const uint32_t* src_k; const int32_t* src_v;
-  uint32_t* dst_k; int32_t* dst_v;
-};
-__device__ __forceinline__ PassIo pass_io(const SortBuffers& buf, int32_t* idx_out, int pass, long long seg_off) {
-  PassIo io;
-  io.src_k = ((pass == 2) ? buf.keys_b : buf.keys_a) + seg_off;
-  io.src_v = ((pass == 2) ? buf.vals_b : buf.vals_a) + seg_off;
-  io.dst_k = ((pass == 0 || pass == 2) ? buf.keys_a : buf.keys_b) + seg_off;
-  io.dst_v = ((pass == 0 || pass == 2) ? buf.vals_a : (pass == 3 ? idx_out : buf.vals_b)) + seg_off;
-  return io;
-}
-
-// counts[seg][tile][digit]: how many elements of the tile have that digit in this pass.
-__global__ void __launch_bounds__(kSortThreads, 4)
-sort_count_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
-                  uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
-  __shared__ uint32_t hist[kRadix];
-  grid_dependency_wait();
-  const long long seg = blockIdx.x / tiles;
-  const int tile = (int)(blockIdx.x - seg * tiles);
-  const PassIo io = pass_io(buf, idx_out, pass, seg * N);
-  const float* s_in = scores + seg * N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t lt_mask = (1u << lane) - 1u;
-  const int shift = 8 * pass;
-  for (int i = tid; i < kRadix; i += kSortThreads) hist[i] = 0;
-  __syncthreads();
-  // counting does not care about the order inside the tile: where the segment allows 16-byte
-  // loads, a thread takes 8 consecutive elements with two of them
-  const long long w0 = (long long)tile * kTileItems + (long long)warp * kWarpItems;
-  const uint32_t* base = pass == 0 ? reinterpret_cast<const uint32_t*>(s_in) : io.src_k;
-  const bool wide = (reinterpret_cast<uintptr_t>(base) & 15u) == 0 && w0 + kWarpItems <= N;
-  uint32_t keys[kItems];
-  if (wide) {
-    const uint4* src = reinterpret_cast<const uint4*>(base) + (w0 >> 2) + lane * 2;
-    const uint4 a = src[0], b = src[1];
-    keys[0] = a.x; keys[1] = a.y; keys[2] = a.z; keys[3] = a.w;
-    keys[4] = b.x; keys[5] = b.y; keys[6] = b.z; keys[7] = b.w;
-    if (pass == 0) {
-#pragma unroll
-      for (int k = 0; k < kItems; ++k) keys[k] = score_to_key(__uint_as_float(keys[k]));
-    }
-  }
-#pragma unroll
-  for (int k = 0; k < kItems; ++k) {
-    const long long i = w0 + k * 32 + lane;
-    const bool valid = wide || i < N;
-    uint32_t key = 0;
-    if (wide) key = keys[k];
-    else if (valid) key = (pass == 0) ? score_to_key(s_in[i]) : io.src_k[i];
-    const uint32_t digit = (key >> shift) & 0xffu;
-    if (pass < 3) {
-      // the low digits are spread over their 256 bins: plain shared-memory atomics hardly collide
-      if (valid) atomicAdd(&hist[digit], 1u);
-    } else {
-      // the top digit (sign and high exponent bits) takes a handful of values: add up per warp first
-      const uint32_t peers = same_digit_lanes(digit, valid);
-      if (valid && (peers & lt_mask) == 0) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
-    }
-  }
-  __syncthreads();
-  for (int i = tid; i < kRadix; i += kSortThreads) counts[((long long)seg * tiles + tile) * kRadix + i] = hist[i];
-}
-
-// One tile of one pass: stable scatter.  Inside a tile the order is (warp, item, lane), which
-// is the order of the positions.
-__global__ void __launch_bounds__(kSortThreads, 2)
-sort_scatter_kernel(const float* __restrict__ scores, SortBuffers buf, int32_t* idx_out,
-                    const uint32_t* __restrict__ counts, long long N, int tiles, int pass) {
-  __shared__ uint32_t tile_base[kRadix];          // first output position of every digit for this tile
-  __shared__ uint32_t tile_start[kRadix];         // first slot of every digit inside the reordered tile
-  __shared__ uint16_t warp_cnt[kWarps][kRadix];   // count, then exclusive offset, per (warp, digit)
-  __shared__ uint32_t scan_tmp[2][kRadix / 32];
-  __shared__ uint32_t stage_k[kTileItems];        // the tile, reordered by digit, before it goes out
-  __shared__ int32_t stage_v[kTileItems];
-
-  grid_dependency_wait();
-  const long long seg = blockIdx.x / tiles;
-  const int tile = (int)(blockIdx.x - seg * tiles);
-  const PassIo io = pass_io(buf, idx_out, pass, seg * N);
-  const float* s_in = scores + seg * N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t lt_mask = (1u << lane) - 1u;
-  const int shift = 8 * pass;
-  const long long t0 = (long long)tile * kTileItems;
-
-  // ---- the tile's elements (issued first: the loads are in flight during the prologue)
-  uint32_t key[kItems]; int32_t val[kItems]; uint32_t rank[kItems];
-  {
-    const long long w0 = t0 + (long long)warp * kWarpItems;
-#pragma unroll
-    for (int k = 0; k < kItems; ++k) {
-      const long long i = w0 + k * 32 + lane;
-      key[k] = 0; val[k] = -1;
-      if (i < N) {
-        if (pass == 0) { key[k] = score_to_key(s_in[i]); val[k] = (int32_t)i; }
-        else { key[k] = io.src_k[i]; val[k] = io.src_v[i]; }
-      }
-    }
-  }
-
-  // ---- where the tile's digits go: (elements of smaller digits in the whole segment) +
-  //      (elements of the same digit in earlier tiles); and where they sit inside the tile
-  uint32_t total = 0, before = 0, mine = 0, incl_t = 0, incl_m = 0;
-  if (tid < kRadix) {
-    const uint32_t* c = counts + (long long)seg * tiles * kRadix + tid;
-    for (int t = 0; t < tiles; ++t) {
-      const uint32_t v = c[(long long)t * kRadix];
-      total += v;
-      if (t < tile) before += v;
-      if (t == tile) mine = v;
-    }
-    incl_t = total; incl_m = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t a = __shfl_up_sync(0xffffffffu, incl_t, o);
-      const uint32_t b2 = __shfl_up_sync(0xffffffffu, incl_m, o);
-      if (lane >= o) { incl_t += a; incl_m += b2; }
-    }
-    if (lane == 31) { scan_tmp[0][warp] = incl_t; scan_tmp[1][warp] = incl_m; }
-  }
-  // this warp's counters, then the rank of every element among the warp's elements of its digit
-  for (int dgt = lane; dgt < kRadix; dgt += 32) warp_cnt[warp][dgt] = 0;
-  __syncwarp();
-#pragma unroll
-  for (int k = 0; k < kItems; ++k) {
-    const bool valid = val[k] >= 0;
-    const uint32_t digit = (key[k] >> shift) & 0xffu;
-    const uint32_t peers = same_digit_lanes(digit, valid);
-    uint32_t seen = 0;
-    if (valid) seen = warp_cnt[warp][digit];
-    __syncwarp();
-    if (valid && (peers & lt_mask) == 0) warp_cnt[warp][digit] = (uint16_t)(seen + __popc(peers));
-    __syncwarp();
-    rank[k] = seen + __popc(peers & lt_mask);
-  }
-  __syncthreads();
-  if (tid < kRadix) {
-    uint32_t add_t = 0, add_m = 0;
-    for (int wv = 0; wv < warp; ++wv) { add_t += scan_tmp[0][wv]; add_m += scan_tmp[1][wv]; }
-    tile_base[tid] = incl_t - total + add_t + before;
-    tile_start[tid] = incl_m - mine + add_m;
-    // per digit: exclusive scan over the warps
-    uint32_t run = 0;
-#pragma unroll
-    for (int wv = 0; wv < kWarps; ++wv) {
-      const uint32_t cnt = warp_cnt[wv][tid];
-      warp_cnt[wv][tid] = (uint16_t)run;
-      run += cnt;
-    }
-  }
-  __syncthreads();
-  // ---- reorder the tile by digit in shared memory ...
-#pragma unroll
-  for (int k = 0; k < kItems; ++k) {
-    if (val[k] >= 0) {
-      const uint32_t digit = (key[k] >> shift) & 0xffu;
-      const uint32_t slot = tile_start[digit] + warp_cnt[warp][digit] + rank[k];
-      stage_k[slot] = key[k];
-      stage_v[slot] = val[k];
-    }
-  }
-  __syncthreads();
-  // ---- ... and write it out: neighbouring threads hold neighbours of the same digit, so the
-  //      stores of a warp fall into a few contiguous runs
-  const int n_tile = (int)min((long long)kTileItems, N - t0);
-#pragma unroll
-  for (int k = 0; k < kItems; ++k) {
-    const int slot = k * kSortThreads + tid;
-    if (slot < n_tile) {
-      const uint32_t kk = stage_k[slot];
-      const uint32_t digit = (kk >> shift) & 0xffu;
-      const uint32_t pos = tile_base[digit] + ((uint32_t)slot - tile_start[digit]);
-      io.dst_k[pos] = kk;
-      io.dst_v[pos] = stage_v[slot];
-    }
-  }
-}
 
 // ---------------------------------------------------------------------------------------------
 // Segments of at most kSegMaxN elements: one CTA sorts one whole segment inside its SM.
@@ -338,7 +124,13 @@ __device__ __forceinline__ void seg_for_keys(const float* s_in, int N, int tid, 
 template <int T>
 __global__ void __launch_bounds__(T, T == 1024 ? 1 : 4)
 segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ keys_out,
-                    int32_t* __restrict__ idx_out, int N) {
+                    int32_t* __restrict__ idx_out, long long seg_len, int chunks) {
+  // CTA x sorts chunk x % chunks of segment x / chunks: the positions from chunk * kSegMaxN on (a segment of
+  // up to kSegMaxN elements is one chunk; the chunks of a longer one are merged afterwards)
+  const long long seg = blockIdx.x / (unsigned)chunks;
+  const int chunk = (int)(blockIdx.x - seg * chunks);
+  const long long first = seg * seg_len + (long long)chunk * kSegMaxN;      // of this chunk, in all three arrays
+  const int N = (int)min((long long)kSegMaxN, seg_len - (long long)chunk * kSegMaxN);
   constexpr int kRowShift = (T == 1024) ? 12 : 10;          // log2 of a row of counters in bytes
   static_assert(T == 1024 || T == 256, "row shift");
   constexpr int kScanWarps = T / 64;                        // the scan runs on the first T / 2 threads
@@ -358,7 +150,7 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
   const uint32_t cbase = cnt + (uint32_t)(tid ^ (((tid >> 5) & 3) << 2)) * 4u;
 
   grid_dependency_wait();
-  const float* s_in = scores + (long long)blockIdx.x * N;
+  const float* s_in = scores + first;
 
   // ---- the keys, once; the identity as the first order; which bits differ anywhere in the segment
   uint32_t diff = 0;
@@ -517,12 +309,115 @@ segment_sort_kernel(const float* __restrict__ scores, uint32_t* __restrict__ key
   }
 
   // ---- out: the positions (a slot's position is key_slot of it: the map is its own inverse), and the keys
-  uint32_t* k_out = keys_out + (long long)blockIdx.x * N;
-  int32_t* i_out = idx_out + (long long)blockIdx.x * N;
+  uint32_t* k_out = keys_out + first;
+  int32_t* i_out = idx_out + first;
+  const int pos0 = chunk * kSegMaxN;
   for (int j = tid; j < N; j += T) {
     const uint32_t q = lds_u16(perm + place_slot((uint32_t)j) * 2u);
-    i_out[j] = (int32_t)key_slot(q);
+    i_out[j] = pos0 + (int32_t)key_slot(q);
     k_out[j] = lds_u32(keys + q * 4u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Segments longer than kSegMaxN: their chunks come sorted from segment_sort_kernel and are merged
+// pairwise, level by level (runs of kSegMaxN << level elements).  A CTA produces kMergeTile
+// consecutive outputs of one pair of runs A, B: it finds where the tile's first and last output
+// split between A and B (the merge path: a binary search over one diagonal each), brings the two
+// stretches into shared memory, and every thread merges kMergeItems consecutive outputs from its
+// own diagonal.  Equal keys are taken from A first: A holds the smaller positions and both runs
+// are stable, so the merged run is in (key, position) order as well.
+constexpr int kMergeThreads = 512;
+constexpr int kMergeItems = 8;
+constexpr int kMergeTile = kMergeThreads * kMergeItems;       // 4096; divides kSegMaxN
+
+// Number of elements taken from A among the first `diag` outputs of merging A (na) and B (nb).
+__device__ __forceinline__ int merge_path(int diag, int na, int nb, const uint32_t* a, const uint32_t* b) {
+  int lo = max(0, diag - nb), hi = min(diag, na);
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    // A[mid] is among the first diag outputs iff it does not come after B[diag - 1 - mid]
+    if (a[mid] <= b[diag - 1 - mid]) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+// The same by one warp over global memory, 32 probes per round (a round trip per round, not per probe).
+__device__ __forceinline__ int merge_path_warp(int diag, int na, int nb, const uint32_t* __restrict__ a,
+                                               const uint32_t* __restrict__ b) {
+  const int lane = threadIdx.x & 31;
+  int lo = max(0, diag - nb), hi = min(diag, na);          // the answer lies in [lo, hi]
+  while (hi > lo) {
+    const int step = (hi - lo + 31) / 32;
+    const int i = lo + (lane + 1) * step - 1;              // this lane's probe
+    bool before = false;                                   // "A[i] is among the first diag outputs": true for a prefix of the probes
+    if (i < hi) before = a[i] <= b[diag - 1 - i];
+    const int n_before = __popc(__ballot_sync(0xffffffffu, before));
+    const int new_lo = n_before == 0 ? lo : min(hi, lo + n_before * step);
+    const int new_hi = n_before == 32 ? hi : min(hi, lo + (n_before + 1) * step - 1);
+    lo = new_lo;
+    hi = new_hi;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(kMergeThreads)
+merge_runs_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ vals_in,
+                  uint32_t* __restrict__ keys_out, int32_t* __restrict__ vals_out, long long seg_len, long long run,
+                  int tiles_per_seg) {
+  __shared__ uint32_t s_key[kMergeTile];
+  __shared__ int32_t s_val[kMergeTile];
+  __shared__ int s_split[2];
+  grid_dependency_wait();
+  const long long seg = blockIdx.x / (unsigned)tiles_per_seg;
+  const long long t0 = (long long)(blockIdx.x - seg * tiles_per_seg) * kMergeTile;    // first output, inside the segment
+  const long long pair0 = t0 / (2 * run) * (2 * run);                                  // where this tile's pair of runs starts
+  const int na = (int)min(run, seg_len - pair0);
+  const int nb = (int)max(0LL, min(run, seg_len - pair0 - run));
+  const long long base = seg * seg_len + pair0;
+  const uint32_t* ka = keys_in + base;
+  const uint32_t* kb = ka + na;
+  const int d0 = (int)(t0 - pair0);
+  const int d1 = min(d0 + kMergeTile, na + nb);
+  const int tid = threadIdx.x;
+  if (tid < 64) {                                          // warp 0: the tile's first output; warp 1: one past its last
+    const int split = merge_path_warp(tid < 32 ? d0 : d1, na, nb, ka, kb);
+    if ((tid & 31) == 0) s_split[tid >> 5] = split;
+  }
+  __syncthreads();
+  const int a0 = s_split[0], a1 = s_split[1];
+  const int b0 = d0 - a0, b1 = d1 - a1;
+  const int ca = a1 - a0, cb = b1 - b0;                   // this tile's elements of A, then of B, in shared memory
+  for (int i = tid; i < ca + cb; i += kMergeThreads) {
+    const long long src = base + (i < ca ? (long long)a0 + i : (long long)na + b0 + (i - ca));
+    s_key[i] = keys_in[src];
+    s_val[i] = vals_in[src];
+  }
+  __syncthreads();
+  const int n_out = d1 - d0;
+  const int my0 = min(tid * kMergeItems, n_out);
+  int ia = merge_path(my0, ca, cb, s_key, s_key + ca);
+  int ib = my0 - ia;
+  uint32_t ok[kMergeItems]; int32_t ov[kMergeItems];
+#pragma unroll
+  for (int k = 0; k < kMergeItems; ++k) {
+    const bool has_a = ia < ca, has_b = ib < cb;
+    const uint32_t xa = has_a ? s_key[ia] : 0xffffffffu, xb = has_b ? s_key[ca + ib] : 0xffffffffu;
+    const bool take_a = has_a && (!has_b || xa <= xb);
+    ok[k] = take_a ? xa : xb;
+    ov[k] = take_a ? s_val[ia] : (has_b ? s_val[ca + ib] : 0);
+    if (take_a) ++ia; else ++ib;
+  }
+  __syncthreads();                                         // everyone has read its inputs: the buffers take the outputs
+#pragma unroll
+  for (int k = 0; k < kMergeItems; ++k) {
+    if (my0 + k < n_out) { s_key[my0 + k] = ok[k]; s_val[my0 + k] = ov[k]; }
+  }
+  __syncthreads();
+  const long long dst = base + d0;
+  for (int i = tid; i < n_out; i += kMergeThreads) {
+    keys_out[dst + i] = s_key[i];
+    vals_out[dst + i] = s_val[i];
   }
 }
 
@@ -577,17 +472,24 @@ static kvc_status segment_sort_prepare(long long N, int* threads) {
   return KVC_OK;
 }
 
-static int sort_tiles(const Problem& P) { return (int)((P.N + kTileItems - 1) / kTileItems); }
-
-size_t compose_workspace_bytes(const Problem& P) {
-  const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
-  const size_t segments = (size_t)P.L * P.Bt * P.Hkv;
-  return 4 * align_up(items * 4) + align_up(segments * sort_tiles(P) * kRadix * sizeof(uint32_t));
+// Scratch of the ranking: the sorted keys [L, Bt, Hkv, N] and, for segments of several chunks, one more
+// buffer of keys and one of positions for the merge levels to alternate with (keys, idx).
+struct SortRegions {
+  size_t keys_a, vals_a, keys_b, total;
+};
+static SortRegions sort_regions(const Problem& P) {
+  const size_t region = align_up((size_t)P.L * P.Bt * P.Hkv * P.N * 4);
+  SortRegions r;
+  if (P.N <= kSegMaxN) { r.keys_a = r.vals_a = 0; r.keys_b = 0; r.total = region; }
+  else { r.keys_a = 0; r.vals_a = region; r.keys_b = 2 * region; r.total = 3 * region; }
+  return r;
 }
+
+size_t compose_workspace_bytes(const Problem& P) { return sort_regions(P).total; }
 
 kvc_status launch_sorted_scores(const Problem& P, const void* ws, float* sorted, cudaStream_t st) {
   const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
-  const uint32_t* keys_b = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(ws) + 2 * align_up(items * 4));
+  const uint32_t* keys_b = reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(ws) + sort_regions(P).keys_b);
   KVC_CUDA(launch_dependent(sorted_scores_kernel, dim3((unsigned)((items + 255) / 256)), dim3(256), 0, st,
                             keys_b, sorted, (long long)items));
   KVC_LAUNCH_CHECK("sorted_scores_kernel");
@@ -600,52 +502,62 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
     set_error("compose: workspace too small");
     return KVC_ERR_WORKSPACE;
   }
-  const size_t items = (size_t)P.L * P.Bt * P.Hkv * P.N;
-  const size_t region = align_up(items * 4);
   char* w = reinterpret_cast<char*>(ws);
-  SortBuffers buf;
-  buf.keys_a = reinterpret_cast<uint32_t*>(w);
-  buf.vals_a = reinterpret_cast<int32_t*>(w + region);
-  buf.keys_b = reinterpret_cast<uint32_t*>(w + 2 * region);
-  buf.vals_b = reinterpret_cast<int32_t*>(w + 3 * region);
-  uint32_t* counts = reinterpret_cast<uint32_t*>(w + 4 * region);
+  const SortRegions reg = sort_regions(P);
+  uint32_t* const keys_a = reinterpret_cast<uint32_t*>(w + reg.keys_a);
+  int32_t* const vals_a = reinterpret_cast<int32_t*>(w + reg.vals_a);
+  uint32_t* const keys_b = reinterpret_cast<uint32_t*>(w + reg.keys_b);
   const long long segments = (long long)P.L * P.Bt * P.Hkv;
   int seg_threads = 0;
-  const kvc_status seg_state = segment_sort_prepare(P.N, &seg_threads);
+  const long long chunk_len = P.N < kSegMaxN ? P.N : (long long)kSegMaxN;
+  const kvc_status seg_state = segment_sort_prepare(chunk_len, &seg_threads);
   if (seg_state != KVC_OK && seg_state != KVC_ERR_UNSUPPORTED) return seg_state;
-  const int tiles = sort_tiles(P);
-  const long long blocks = segments * tiles;
-  if (seg_state == KVC_OK) {
-    // a segment fits one SM's shared memory: the whole sort in one launch, one CTA per segment
-    if (segments >= (1LL << 31)) {
+  if (seg_state != KVC_OK) {
+    set_error("compose: this device cannot give a CTA the %zu bytes of shared memory the ranking needs",
+              (size_t)seg_layout(chunk_len, chunk_len > 8192 ? 1024 : 256).total);
+    return KVC_ERR_UNSUPPORTED;
+  }
+  {
+    // Chunks of up to kSegMaxN elements are sorted inside one SM each: a whole segment in one launch, or,
+    // for longer segments, its chunks, which are then merged pairwise, level by level.  The levels
+    // alternate between (keys_a, vals_a) and (keys_b, idx); the last one has to end in the latter.
+    const long long chunks = (P.N + kSegMaxN - 1) / kSegMaxN;
+    int levels = 0;
+    while ((1LL << levels) < chunks) ++levels;
+    const long long merge_tiles = (P.N + kMergeTile - 1) / kMergeTile;
+    if (segments * chunks >= (1LL << 31) || segments * merge_tiles >= (1LL << 31)) {
       set_error("compose: too many segments");
       return KVC_ERR_UNSUPPORTED;
     }
-    const size_t smem = seg_layout(P.N, seg_threads).total;
+    bool in_b = (levels % 2) == 0;                 // where the sorted chunks go
+    uint32_t* k_cur = in_b ? keys_b : keys_a;
+    int32_t* v_cur = in_b ? idx : vals_a;
+    const size_t smem = seg_layout(chunk_len, seg_threads).total;
+    const unsigned grid = (unsigned)(segments * chunks);
     if (seg_threads == 1024) {
-      KVC_CUDA(launch_dependent(segment_sort_kernel<1024>, dim3((unsigned)segments), dim3(1024), smem, st,
-                                scores, buf.keys_b, idx, (int)P.N));
+      KVC_CUDA(launch_dependent(segment_sort_kernel<1024>, dim3(grid), dim3(1024), smem, st,
+                                scores, k_cur, v_cur, P.N, (int)chunks));
     } else {
-      KVC_CUDA(launch_dependent(segment_sort_kernel<256>, dim3((unsigned)segments), dim3(256), smem, st,
-                                scores, buf.keys_b, idx, (int)P.N));
+      KVC_CUDA(launch_dependent(segment_sort_kernel<256>, dim3(grid), dim3(256), smem, st,
+                                scores, k_cur, v_cur, P.N, (int)chunks));
     }
     KVC_LAUNCH_CHECK("segment_sort_kernel");
-  } else if (blocks >= (1LL << 31)) {
-    set_error("compose: too many sort tiles");
-    return KVC_ERR_UNSUPPORTED;
-  }
-  for (int pass = 0; pass < 4 && seg_state != KVC_OK; ++pass) {
-    KVC_CUDA(launch_dependent(sort_count_kernel, dim3((unsigned)blocks), dim3(kSortThreads), 0, st,
-                              scores, buf, idx, counts, P.N, tiles, pass));
-    KVC_LAUNCH_CHECK("sort_count_kernel");
-    KVC_CUDA(launch_dependent(sort_scatter_kernel, dim3((unsigned)blocks), dim3(kSortThreads), 0, st,
-                              scores, buf, idx, counts, P.N, tiles, pass));
-    KVC_LAUNCH_CHECK("sort_scatter_kernel");
+    for (int level = 0; level < levels; ++level) {
+      in_b = !in_b;
+      uint32_t* k_nxt = in_b ? keys_b : keys_a;
+      int32_t* v_nxt = in_b ? idx : vals_a;
+      KVC_CUDA(launch_dependent(merge_runs_kernel, dim3((unsigned)(segments * merge_tiles)), dim3(kMergeThreads), 0, st,
+                                (const uint32_t*)k_cur, (const int32_t*)v_cur, k_nxt, v_nxt, P.N,
+                                (long long)kSegMaxN << level, (int)merge_tiles));
+      KVC_LAUNCH_CHECK("merge_runs_kernel");
+      k_cur = k_nxt;
+      v_cur = v_nxt;
+    }
   }
   if (composite == nullptr) return KVC_OK;      // ranking only (the unstructured variant has no Eq. 19)
   const long long total = (long long)P.L * P.Bt * P.N;
   KVC_CUDA(launch_dependent(compose_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                            buf.keys_b, composite, P.Hkv, P.N, total, P.agg_head));
+                            keys_b, composite, P.Hkv, P.N, total, P.agg_head));
   KVC_LAUNCH_CHECK("compose_kernel");
   return KVC_OK;
 }

@@ -341,12 +341,12 @@ def test_exact_ties_are_broken_by_position_and_layer():
 
 
 @pytest.mark.parametrize("N", [1, 2, 31, 33, 255, 257, 400, 1000, 4095, 4097, 8191, 8192, 8193, 12345,
-                               32767, 32768, 32769, 40000])
+                               32767, 32768, 32769, 40000, 65536, 70000, 131072, 200000])
 def test_ranking_alone_across_lengths_and_both_sorts(N):
     """Eqs. 17-19 on scores given by the caller: lengths on both sides of every switch of the
-    ranking (places per thread, CTA size, one SM per segment or all segments over tiles), segments
-    that do not start on 16 bytes, and values of every kind -- long runs of equal scores, both
-    zeros, negatives, denormals, huge values."""
+    ranking (places per thread, CTA size, one chunk per segment or several that are merged over one,
+    two and three levels, a last chunk of any length), segments that do not start on 16 bytes, and
+    values of every kind -- long runs of equal scores, both zeros, negatives, denormals, huge values."""
     dev = _cuda()
     L, Hkv = 2, 3
     cfg = W.WorkloadConfig("rank", L, Hkv, Hkv, 64, N, 1, dtype="f32", elem_std=1.0)
