@@ -113,17 +113,36 @@ select_hist_kernel(const float* __restrict__ composite, unsigned int* __restrict
     long long i = t0 + threadIdx.x;
     long long r = i / M, kk = i - r * M;
     long long base = row_start(r, b, Bt, hpr, N) + floor;      // (recomputed only when the row changes)
-#pragma unroll 4
+    // all of the thread's loads first ...
+    float v[kItemsPerThread];
+#pragma unroll
     for (int it = 0; it < kItemsPerThread; ++it) {
-      if (i < total) {
-        const uint32_t key = score_to_key(composite[base + kk]);
-        if ((key & hi_mask) == prefix) atomicAdd(&sh[(key >> shift) & 0xffu], 1u);
-      }
+      v[it] = 0.f;
+      if (i < total) v[it] = composite[base + kk];
       i += kHistThreads;
       kk += kHistThreads;
       if (kk >= M) {
         while (kk >= M) { kk -= M; ++r; }
         base = row_start(r, b, Bt, hpr, N) + floor;
+      }
+    }
+    // ... then the bins.  Consecutive lanes hold consecutive entries of a non-increasing row: equal digits
+    // come in runs, and only the first lane of a run adds (its length) to the bin.
+    i = t0 + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int it = 0; it < kItemsPerThread; ++it, i += kHistThreads) {
+      uint32_t digit = 0x100u;                                  // not in the bucket / beyond the pool
+      if (i < total) {
+        const uint32_t key = score_to_key(v[it]);
+        if ((key & hi_mask) == prefix) digit = (key >> shift) & 0xffu;
+      }
+      const uint32_t prev = __shfl_up_sync(0xffffffffu, digit, 1);
+      const bool head = lane == 0 || prev != digit;
+      const uint32_t heads = __ballot_sync(0xffffffffu, head);
+      if (head && digit < 0x100u) {
+        const uint32_t later = lane == 31 ? 0u : (heads >> (lane + 1));
+        atomicAdd(&sh[digit], (unsigned int)(later ? __ffs(later) : 32 - lane));
       }
     }
   }
