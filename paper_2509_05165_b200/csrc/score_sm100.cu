@@ -85,7 +85,8 @@ constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // 2 s: far 
 constexpr int kMaxFastLayers = 112;   // 2 tensor maps per layer must fit the 32 KB kernel-parameter space
 
 struct FastParams {
-  CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (d, N, Hkv, Bt), box 64 x 128 x 1 x 1, 128-byte swizzle
+  CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (64, N, d / 64, Hkv, Bt), box 64 x 128 x d / 64 x 1 x 1, 128-byte swizzle:
+                                        // a tile arrives as d / 64 blocks of 128 rows of 128 bytes with one copy
   CUtensorMap q_maps[kMaxFastLayers];   // Q^(l) as (d, w, Hq, Bt), box 64 x w x G x 1
   float4* partial;             // [U][RPU][64]: (ref, sum) of rows 2i and 2i+1 of one run
   float4* group_partial;       // [U][NG][64]: the same, folded over a group of runs
@@ -191,9 +192,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
-               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4, unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -952,8 +960,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       auto prefetch_next = [&]() {
         if (ahead_pos >= my_tiles) return;
         if (ahead.valid(P)) {
-          for (int hf = 0; hf < SL::kHalves; ++hf)
-            tma_prefetch_4d(P.k_maps + ahead.l, hf * 64, ahead.tile(P) * kTile, ahead.h, ahead.b);
+          tma_prefetch_5d(P.k_maps + ahead.l, 0, ahead.tile(P) * kTile, 0, ahead.h, ahead.b);
         }
         ahead.advance(P);
         ++ahead_pos;
@@ -981,9 +988,9 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             if (ok) {
               mbar_expect_tx(bar_kfull(kr.i), SL::kTileBytes);
               // pass 1 leaves the rows in L2 for pass 2; pass 2 is their last use
-              for (int hf = 0; hf < SL::kHalves; ++hf)
-                tma_load_4d(sbase + SL::kK + kr.i * SL::kTileBytes + hf * (kTile * 128), P.k_maps + c.l,
-                            bar_kfull(kr.i), hf * 64, c.tile(P) * kTile, c.h, c.b, pass == 0 ? pol_keep : pol_stream);
+              // (one copy for the whole tile: the 64-element halves of the rows are a dimension of the map)
+              tma_load_5d(sbase + SL::kK + kr.i * SL::kTileBytes, P.k_maps + c.l, bar_kfull(kr.i), 0, c.tile(P) * kTile, 0,
+                          c.h, c.b, pass == 0 ? pol_keep : pol_stream);
               kr.next(SL::kStages);
               if (nk < SL::kStages) ++nk;
             }
@@ -1174,14 +1181,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-bool encode_map(CUtensorMap* m, const void* base, const long long dims[4], const long long strides_bytes[3],
-                const unsigned box[4]) {
+bool encode_map(CUtensorMap* m, const void* base, int rank, const long long* dims, const long long* strides_bytes,
+                const unsigned* box) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  cuuint64_t gd[4]; cuuint64_t gs[3]; cuuint32_t bx[4]; cuuint32_t es[4] = {1, 1, 1, 1};
-  for (int i = 0; i < 4; ++i) { gd[i] = (cuuint64_t)dims[i]; bx[i] = box[i]; }
-  for (int i = 0; i < 3; ++i) gs[i] = (cuuint64_t)strides_bytes[i];
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs, bx, es,
+  cuuint64_t gd[5]; cuuint64_t gs[4]; cuuint32_t bx[5]; cuuint32_t es[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gd[i] = (cuuint64_t)dims[i]; bx[i] = box[i]; }
+  for (int i = 0; i < rank - 1; ++i) gs[i] = (cuuint64_t)strides_bytes[i];
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1328,14 +1335,14 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   const int G = P.Hq / P.Hkv;
   static thread_local FastParams fp;
   for (int l = 0; l < P.L; ++l) {
-    const long long kd[4] = {P.d, P.N, P.Hkv, P.Bt};
-    const long long ks[3] = {P.kvs[2] * 2, P.kvs[1] * 2, P.kvs[0] * 2};
-    const unsigned kb[4] = {64, (unsigned)kTile, 1, 1};
+    const long long kd[5] = {64, P.N, P.d / 64, P.Hkv, P.Bt};
+    const long long ks[4] = {P.kvs[2] * 2, 128, P.kvs[1] * 2, P.kvs[0] * 2};
+    const unsigned kb[5] = {64, (unsigned)kTile, (unsigned)(P.d / 64), 1, 1};
     const long long qd[4] = {P.d, P.w, P.Hq, P.Bt};
     const long long qs[3] = {P.qs[2] * 2, P.qs[1] * 2, P.qs[0] * 2};
     const unsigned qb[4] = {64, (unsigned)(pl.CH == 1 ? P.w : kRows), (unsigned)pl.HPT, 1};
-    if (!encode_map(&fp.k_maps[l], k.p[l], kd, ks, kb)) return KVC_ERR_UNSUPPORTED;
-    if (!encode_map(&fp.q_maps[l], q.p[l], qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
+    if (!encode_map(&fp.k_maps[l], k.p[l], 5, kd, ks, kb)) return KVC_ERR_UNSUPPORTED;
+    if (!encode_map(&fp.q_maps[l], q.p[l], 4, qd, qs, qb)) return KVC_ERR_UNSUPPORTED;
   }
   char* w = reinterpret_cast<char*>(ws);
 
