@@ -197,3 +197,29 @@ def test_unstructured_variant_with_value_norm_weighting():
     Pz.assert_scores_close(S, _oracle_vnorm_scores(wl, desc))
     n_ref, off_ref = oracle.select_unstructured(S[:, 0].astype(np.float64), B)
     assert np.array_equal(n_ref, _host(n_keep)[0]) and np.array_equal(off_ref, _host(off)[0])
+
+
+def test_unstructured_selection_on_segments_of_several_chunks():
+    """The per-head selection of App. A.2 on scores given by the caller, with heads long enough that the
+    ranking sorts them in chunks and merges: the sorted scores the selection reads then sit behind the
+    merge buffers in the workspace."""
+    import oracle
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    dev = torch.device("cuda:0")
+    L, Hkv, N = 2, 2, 40000
+    cfg = W.WorkloadConfig("unstructured_long", L, Hkv, Hkv, 64, N, 1, dtype="f32", elem_std=1.0)
+    desc = kvc.desc_from_config(cfg)
+    g = np.random.default_rng(7)
+    S = (np.round(g.random((L, 1, Hkv, N)) * 4096) / 4096).astype(np.float32)          # many exact ties
+    scores = torch.from_numpy(S).to(dev)
+    B = int(0.3 * L * Hkv * N)
+    idx = torch.empty((L, 1, Hkv, N), dtype=torch.int32, device=dev)
+    n_keep = torch.empty((1, L, Hkv), dtype=torch.int32, device=dev)
+    off = torch.empty((1, L * Hkv + 1), dtype=torch.int64, device=dev)
+    ws = torch.empty(kvc.kvc_workspace_size(desc, 0), dtype=torch.uint8, device=dev)
+    kvc.kvc_select_unstructured(desc, scores, B, idx, n_keep, off, ws)
+    torch.cuda.synchronize()
+    Pz.assert_rank_exact(S, _host(idx))
+    n_ref, off_ref = oracle.select_unstructured(S[:, 0].astype(np.float64), B)
+    assert np.array_equal(n_ref, _host(n_keep)[0]) and np.array_equal(off_ref, _host(off)[0])
