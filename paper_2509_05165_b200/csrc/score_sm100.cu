@@ -13,16 +13,15 @@
 //                        reference, converted to fixed point (2^-20) and added, together with an
 //                        arrival count in the top byte, with one integer reduction.  Integer
 //                        addition makes the total independent of the order of arrival, and sum
-//                        and count travel in one word, so a reader needs no fence: the word is
-//                        complete when its count equals the unit's runs.  That is two round
+//                        and count travel in one word, so a reader of the sum needs no fence: the
+//                        word is complete when its count equals the unit's runs.  That is two round
 //                        trips to L2 between the last pass-1 tile of a unit and its first pass-2
-//                        tile.  The long way, always taken as well: the run's record of
-//                        (reference, sum) per row goes to global memory and is counted into its
-//                        group of kGroupRuns runs; every group and every unit has a fixed folding
-//                        CTA (round-robin) whose exchange warp waits for the count and folds in
-//                        a fixed order, down to the rows' log-sum-exp.  Pass 2 uses it for the
-//                        rows whose word says that some run's sum did not fit the fixed-point
-//                        range (a token about 14 nats above token 0).
+//                        tile.  The long way, for the rows whose word says that some run's sum did
+//                        not fit the fixed-point range (a token about 14 nats above token 0): every
+//                        run also writes its (reference, sum) of every row to global memory before
+//                        it adds to the word, and adds with release semantics; a pass-2 thread that
+//                        needs them acquires the complete word and folds the unit's records of its
+//                        row in run order (the same order for every reader).
 //   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
 //                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
 //                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
@@ -41,14 +40,14 @@
 // runs than there are CTAs: 38 MB of K at 148 CTAs, which L2 still holds).  A pass-2 tile only
 // ever waits for pass-1 tiles that lie earlier in every CTA's sequence, so the walk cannot
 // deadlock while all CTAs are resident (the host checks that they can be).  Every wait
-// (mbarrier, shared-memory counter or global flag) is bounded; on expiry the kernel records
+// (mbarrier or global word) is bounded; on expiry the kernel records
 // KVC_ERR_TIMEOUT, stops computing and drains.
 //
 // Warp roles (512 threads): warp 0 = TMA producer (K ring, Q ring, L2 prefetch); warp 1 = MMA
 // issuer of pass 1 and TMEM owner; warp 2 = MMA issuer of pass 2 (two issuers: issuing the eight
 // MMAs of a tile takes a thread about 420 clocks, a commit about 50 and every barrier wait
 // about 100 even when it succeeds at once, which together is more than the 512 tensor clocks of
-// the tile, and the tensor pipe would idle meanwhile); warp 3 = statistics exchange; warps 4-7 =
+// the tile, and the tensor pipe would idle meanwhile); warp 3 has no role; warps 4-7 =
 // pass-2 epilogue; warps 8-15 = pass-1 epilogue (two groups of four warps, each takes one half
 // of every tile's columns).
 #include <cuda.h>
@@ -75,7 +74,6 @@ constexpr int kTile = 128;            // tokens per tile = MMA M = MMA N
 constexpr int kFastThreads = 512;
 constexpr int kRows = 128;            // query rows per unit handled by one MMA (R <= 128)
 constexpr int kMinRunTiles = KVC_SCORE_RUN_TILES;   // runs are longer only where a unit would otherwise have more than 255
-constexpr int kGroupRuns = 8;         // runs whose partials are folded together at the first level
 constexpr int kQSlots = 3;
 constexpr int kPrefetch = KVC_SCORE_PREFETCH;
 constexpr float kLog2eF = 1.4426950408889634f;
@@ -88,11 +86,7 @@ struct FastParams {
   CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (64, N, d / 64, Hkv, Bt), box 64 x 128 x d / 64 x 1 x 1, 128-byte swizzle:
                                         // a tile arrives as d / 64 blocks of 128 rows of 128 bytes with one copy
   CUtensorMap q_maps[kMaxFastLayers];   // Q^(l) as (d, w, Hq, Bt), box 64 x w x G x 1
-  float4* partial;             // [U][RPU][64]: (ref, sum) of rows 2i and 2i+1 of one run
-  float4* group_partial;       // [U][NG][64]: the same, folded over a group of runs
-  int* group_counter;          // [U][NG], preset to -1
-  int* unit_counter;           // [U], preset to -1
-  unsigned int* lse2;          // [U][128] fp32 bits, preset to 0xffffffff ("not there yet")
+  float4* partial;             // [U][RPU][64]: the runs' records: (ref, sum) of rows 2i and 2i+1 of one run
   unsigned long long* acc;     // [U][128], preset to 0: per row  arrivals << 56 | overflows << 48 | sum in units
                                // of 2^-20 of 2^(logit - ref[row]), added to by every run of the unit
   const float* ref;            // [U][128]: the row's reference exponent (its scaled logit against token 0)
@@ -103,7 +97,7 @@ struct FastParams {
   int CH;                      // row tiles per query head: 1, or ceil(w / 128) for windows longer than 128 rows
                                // (then HPT = 1 and row tile q holds rows (q % CH) * 128 .. of query head q / CH)
   long long N, q_pos0;
-  int U, NT, RPU, NG, grid;    // units, tiles per unit, runs per unit, groups per unit, CTAs
+  int U, NT, RPU, grid;        // units, tiles per unit, runs per unit, CTAs
   int RT;                      // tiles per run
   int step_u, step_j;          // grid = step_u * RPU + step_j: how a CTA's next run moves (unit, run in unit)
   int step_l, step_b, step_h, step_q;  // step_u = ((step_l * Bt + step_b) * Hkv + step_h) * QT + step_q
@@ -275,16 +269,10 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 __device__ __forceinline__ void named_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ uint32_t ld_relaxed_u32(const unsigned int* p) {
-  uint32_t v;
-  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_relaxed_u32(unsigned int* p, uint32_t v) {
-  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long long v) {
-  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+// (release: what this thread wrote before -- the run's record of the row -- is visible to whoever
+// acquires a value of the word that includes this addition)
+__device__ __forceinline__ void red_add_release_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -296,20 +284,6 @@ __device__ __forceinline__ float lg2(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void red_add_release(int* p, int v) {
-  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ int ld_acquire_s32(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ int atom_add_acq_rel_cta_shared(uint32_t saddr, int v) {
-  int old;
-  asm volatile("atom.acq_rel.cta.shared::cta.add.s32 %0, [%1], %2;" : "=r"(old) : "r"(saddr), "r"(v) : "memory");
-  return old;
-}
-
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart,
 // 8-row groups 1024 B apart; `addr` may be advanced by 32 B per 16-element K step.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t addr) {
@@ -414,8 +388,7 @@ struct SmemLayout {
   static constexpr int kBarMmaDone = kBarQFree + 8 * kQSlots;  // 2 x 8
   static constexpr int kTmemSlot = kBarMmaDone + 16;           // 4 B (+ padding)
   static constexpr int kCtl = kTmemSlot + 8;                   // Ctl, 24 B
-  static constexpr int kFlushed = kCtl + 24;                   // 4 B: warps that have written a run's record
-  static constexpr int kNegLse = (kFlushed + 8 + 15) / 16 * 16;  // 128 floats, read as 16-byte vectors:
+  static constexpr int kNegLse = (kCtl + 24 + 15) / 16 * 16;   // 128 floats, read as 16-byte vectors:
                                                                // -log-sum-exp of the pass-2 unit
   static constexpr int kStats = kNegLse + kRows * 4;           // 128 rows x float2: the upper half's statistics
   static constexpr int kTotal = kStats + kRows * 8;
@@ -439,17 +412,6 @@ __device__ __noinline__ unsigned long long poll_acc_slow(const unsigned long lon
     if ((++spins & 255u) == 0 && give_up(ctl, t0)) break;
   }
   return v;
-}
-
-// Bounded poll of a log-sum-exp slot (the value itself is the flag).
-__device__ __noinline__ uint32_t poll_lse_slow(const unsigned int* src, volatile Ctl* ctl) {
-  const unsigned long long t0 = globaltimer_ns();
-  uint32_t spins = 0, bits;
-  while ((bits = ld_relaxed_u32(src)) == 0xffffffffu) {
-    __nanosleep(100);
-    if ((++spins & 255u) == 0 && give_up(ctl, t0)) break;
-  }
-  return bits;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -589,7 +551,6 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
     ctl->abort = 0;
     ctl->limit_ns = P.wait_limit_ns;
     ctl->grid_status = P.status;
-    *reinterpret_cast<volatile int*>(smem + SL::kFlushed) = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -702,7 +663,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
       }
       if (run_ends) {
         // the two halves of every row meet through shared memory; the lower half's warps write
-        // the run's record and report it to the statistics warp
+        // the run's record of every row and then push its sum
         if (half == 1) *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
         named_bar(3, 256);
         const float2 other = *stage;
@@ -720,15 +681,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
               if (lv < kAccLimitLog2) add += __float2ull_rn(ex2(lv + (float)kAccFracBits));
               else add += kAccOverflow;                                  // the rows' records decide instead
             }
-            red_add_u64(P.acc + (long long)c.u * kRows + row, add);
-          }
-          __syncwarp();
-          if (lane == 0) {
-            // the four warps order their parts of the record through this counter (release /
-            // acquire within the CTA); the last one publishes the whole record with one
-            // device-wide release
-            const int seen = atom_add_acq_rel_cta_shared(sbase + SL::kFlushed, 1);
-            if ((seen & 3) == 3) red_add_release(P.group_counter + (long long)c.u * P.NG + c.j / kGroupRuns, 1);
+            red_add_release_u64(P.acc + (long long)c.u * kRows + row, add);
           }
         }
         mref = -INFINITY; lsum = 0.f;
@@ -770,8 +723,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         score_row = P.scores + ((long long)cu.q * ((long long)P.L * P.Bt * P.Hkv) + cu.kv_unit(P)) * P.N;
         // a new run: its unit's log-sum-exp.  The short way: the row's pushed word, complete once
         // every run of the unit has arrived (fetched a tile or two ago; polled if it was not
-        // complete then).  If a run's sum did not fit, the folded
-        // records decide (the value is its own flag).
+        // complete then).  If a run's sum did not fit, the runs' records decide.
         float lse = 0.f;
         if (ok && trow < rows_u) {
           bool pushed = false;
@@ -787,10 +739,17 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             }
           }
           if (!pushed) {
-            const unsigned int* src = P.lse2 + (long long)cu.u * kRows + trow;
-            uint32_t bits = ld_relaxed_u32(src);
-            if (bits == 0xffffffffu) bits = poll_lse_slow(src, ctl);
-            lse = __uint_as_float(bits);
+            // the long way: all runs have arrived (the count in the word), and each wrote the row's record
+            // before its release; fold the records in run order (the same order for every reader)
+            asm volatile("fence.acq_rel.gpu;" ::: "memory");
+            const float2* rec = reinterpret_cast<const float2*>(P.partial) + (long long)cu.u * P.RPU * kRows + trow;
+            float M = -INFINITY, Ls = 0.f;
+#pragma unroll 4
+            for (int j = 0; j < P.RPU; ++j) {
+              const float2 v = __ldcg(rec + (long long)j * kRows);
+              combine(M, Ls, v.x, v.y);
+            }
+            lse = M + log2f(Ls);
           }
         }
         early_u = -1;
@@ -1014,88 +973,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         mbar_wait_issued(bar_qfull(i2), (uint32_t)ph, ctl);
       }
     }
-  } else if (warp == 3) {
-    // ============================== statistics exchange ========================================
-    // This CTA folds the groups  x, x + grid, ...  (x = blockIdx.x; a group is numbered
-    // unit * NG + group) and the units  x, x + grid, ...   Jobs are taken in the order in which
-    // they become ready anywhere in the grid -- a group before every unit whose last group is
-    // not smaller -- so a wait here only ever depends on jobs that are earlier in that order.
-    // Lane i owns rows 4i .. 4i+3; a record of 128 rows is 64 float4, two per lane.
-    const int n_groups = P.U * P.NG;
-    int gi = blockIdx.x, un = blockIdx.x;             // next group / next unit of this CTA
-    bool ok = my_runs > 0;
-    while (ok && (gi < n_groups || un < P.U)) {
-      const bool take_group = gi < n_groups && (un >= P.U || gi <= (un + 1) * P.NG - 1);
-      const int* counter = take_group ? P.group_counter + gi : P.unit_counter + un;
-      int target;                                     // the counters start at -1
-      if (take_group) {
-        const int g = gi % P.NG;
-        target = min(kGroupRuns, P.RPU - g * kGroupRuns) - 1;
-      } else {
-        target = P.NG - 1;
-      }
-      if (lane == 0) {
-        const unsigned long long t0 = globaltimer_ns();
-        uint32_t spins = 0;
-        while (ld_acquire_s32(counter) != target) {
-          __nanosleep(200);
-          if ((++spins & 63u) == 0 && give_up(ctl, t0)) { ok = false; break; }
-        }
-      }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) break;
-      __threadfence();                                // the records were published before the counts we saw
-      float4 lo = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), hi = lo;
-      if (take_group) {
-        const int u = gi / P.NG, g = gi - u * P.NG;
-        const int members = target + 1;
-        const float4* src = P.partial + ((long long)u * P.RPU + g * kGroupRuns) * 64 + 2 * lane;
-        // four records in flight at a time (this warp runs on a small register budget)
-#pragma unroll 1
-        for (int r0 = 0; r0 < members; r0 += 4) {
-          float4 v[8];
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            if (r0 + r < members) { v[2 * r] = __ldcg(src + (r0 + r) * 64); v[2 * r + 1] = __ldcg(src + (r0 + r) * 64 + 1); }
-          }
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            if (r0 + r < members) {
-              combine(lo.x, lo.y, v[2 * r].x, v[2 * r].y);
-              combine(lo.z, lo.w, v[2 * r].z, v[2 * r].w);
-              combine(hi.x, hi.y, v[2 * r + 1].x, v[2 * r + 1].y);
-              combine(hi.z, hi.w, v[2 * r + 1].z, v[2 * r + 1].w);
-            }
-          }
-        }
-        float4* dst = P.group_partial + (long long)gi * 64 + 2 * lane;
-        dst[0] = lo;
-        dst[1] = hi;
-        __syncwarp();
-        if (lane == 0) {
-          __threadfence();
-          red_add_release(P.unit_counter + u, 1);
-        }
-        gi += P.grid;
-      } else {
-        const float4* src = P.group_partial + (long long)un * P.NG * 64 + 2 * lane;
-#pragma unroll 2
-        for (int r = 0; r < P.NG; ++r) {
-          const float4 v0 = __ldcg(src + r * 64), v1 = __ldcg(src + r * 64 + 1);
-          combine(lo.x, lo.y, v0.x, v0.y);
-          combine(lo.z, lo.w, v0.z, v0.w);
-          combine(hi.x, hi.y, v1.x, v1.y);
-          combine(hi.z, hi.w, v1.z, v1.w);
-        }
-        unsigned int* out = P.lse2 + (long long)un * kRows + 4 * lane;
-        st_relaxed_u32(out + 0, __float_as_uint(lo.x + log2f(lo.y)));
-        st_relaxed_u32(out + 1, __float_as_uint(lo.z + log2f(lo.w)));
-        st_relaxed_u32(out + 2, __float_as_uint(hi.x + log2f(hi.y)));
-        st_relaxed_u32(out + 3, __float_as_uint(hi.z + log2f(hi.w)));
-        un += P.grid;
-      }
-    }
   }
+  // (warp 3 has no role)
 
   // ---------------- teardown ----------------
   tc_fence_before();
@@ -1113,11 +992,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 // 2^(logit - ref) is then at least about 1, so fixed point with 20 fractional bits keeps it.
 // ------------------------------------------------------------------------------------------------
 struct RefParams {
-  int Bt, Hkv, G, HPT, QT, CH, w, d, NG;
+  int Bt, Hkv, G, HPT, QT, CH, w, d;
   unsigned long long* acc;     // [U][128]: cleared here
-  int* group_counter;          // [U][NG], int* unit_counter [U], unsigned* lse2 [U][128]: preset here
-  int* unit_counter;
-  unsigned int* lse2;
   long long qs0, qs1, qs2, kvs0, kvs1;
   float sl2e;
 };
@@ -1126,11 +1002,8 @@ __global__ void __launch_bounds__(kRows)
 score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ ref) {
   grid_dependency_wait();
   const int u = blockIdx.x, row = threadIdx.x;
-  // the unit's exchange state: empty words, counters at -1, log-sum-exp slots "not there yet"
+  // the unit's exchange state: empty words
   P.acc[(long long)u * kRows + row] = 0ull;
-  P.lse2[(long long)u * kRows + row] = 0xffffffffu;
-  if (row < P.NG) P.group_counter[(long long)u * P.NG + row] = -1;
-  if (row == 0) P.unit_counter[u] = -1;
   const int uh = u / P.QT, qt = u - uh * P.QT;
   const int lb = uh / P.Hkv, h = uh - lb * P.Hkv;
   const int l = lb / P.Bt, b = lb - l * P.Bt;
@@ -1194,10 +1067,10 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const long long* dim
 }
 
 struct FastPlan {
-  int U, NT, RPU, NG, grid, RT;
+  int U, NT, RPU, grid, RT;
   int HPT, QT, CH;             // query heads per row tile, row tiles per KV head, row tiles per query head
   long long total_runs, shift;
-  size_t off_partial, off_group, off_sync, sync_bytes, off_parts, off_acc, off_ref, off_total;
+  size_t off_partial, off_parts, off_acc, off_ref, off_total;
 };
 
 // sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
@@ -1217,7 +1090,6 @@ void make_plan(const Problem& P, int sms, FastPlan* pl) {
   pl->RT = kMinRunTiles;
   if ((pl->NT + pl->RT - 1) / pl->RT > 255) pl->RT = (pl->NT + 254) / 255;   // the arrivals of a unit are counted in 8 bits
   pl->RPU = (pl->NT + pl->RT - 1) / pl->RT;
-  pl->NG = (pl->RPU + kGroupRuns - 1) / kGroupRuns;
   pl->total_runs = (long long)pl->U * pl->RPU;
   pl->grid = sms > 0 ? (int)(pl->total_runs < sms ? pl->total_runs : sms) : 1;
   // pass 2 of a run starts once every CTA has been through the rest of the run's unit, at most
@@ -1227,10 +1099,6 @@ void make_plan(const Problem& P, int sms, FastPlan* pl) {
   pl->shift = lag_runs * pl->RT + KVC_SCORE_LAG_TILES;
   size_t off = 0;
   pl->off_partial = off; off += align_up((size_t)pl->total_runs * 64 * sizeof(float4));
-  pl->off_group = off; off += align_up((size_t)pl->U * pl->NG * 64 * sizeof(float4));
-  pl->off_sync = off;      // [U][NG] group counters, [U] unit counters, [U][128] log-sum-exp slots
-  pl->sync_bytes = ((size_t)pl->U * pl->NG + (size_t)pl->U) * sizeof(int) + (size_t)pl->U * kRows * sizeof(float);
-  off += align_up(pl->sync_bytes);
   pl->off_acc = off; off += align_up((size_t)pl->U * kRows * sizeof(unsigned long long));
   pl->off_ref = off; off += align_up((size_t)pl->U * kRows * sizeof(float));
   pl->off_parts = off;         // partial group aggregates [QT][L*Bt*Hkv][N], only with several row tiles
@@ -1347,17 +1215,12 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   char* w = reinterpret_cast<char*>(ws);
 
   fp.partial = reinterpret_cast<float4*>(w + pl.off_partial);
-  fp.group_partial = reinterpret_cast<float4*>(w + pl.off_group);
-  fp.group_counter = reinterpret_cast<int*>(w + pl.off_sync);
-  fp.unit_counter = fp.group_counter + (size_t)pl.U * pl.NG;
-  fp.lse2 = reinterpret_cast<unsigned int*>(fp.unit_counter + pl.U);
   fp.acc = reinterpret_cast<unsigned long long*>(w + pl.off_acc);
   float* ref = reinterpret_cast<float*>(w + pl.off_ref);
   fp.ref = ref;
   {
     RefParams rp;
-    rp.NG = pl.NG; rp.acc = fp.acc; rp.group_counter = fp.group_counter; rp.unit_counter = fp.unit_counter;
-    rp.lse2 = fp.lse2;
+    rp.acc = fp.acc;
     rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.CH = pl.CH; rp.w = P.w; rp.d = P.d;
     rp.qs0 = P.qs[0]; rp.qs1 = P.qs[1]; rp.qs2 = P.qs[2]; rp.kvs0 = P.kvs[0]; rp.kvs1 = P.kvs[1];
     rp.sl2e = P.scale * kLog2eF;
@@ -1373,7 +1236,7 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   fp.L = P.L; fp.Bt = P.Bt; fp.Hkv = P.Hkv; fp.G = G;
   fp.HPT = pl.HPT; fp.QT = pl.QT; fp.CH = pl.CH; fp.w = P.w;
   fp.N = P.N; fp.q_pos0 = P.q_pos0;
-  fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.RT = pl.RT; fp.NG = pl.NG; fp.grid = pl.grid;
+  fp.U = pl.U; fp.NT = pl.NT; fp.RPU = pl.RPU; fp.RT = pl.RT; fp.grid = pl.grid;
   fp.total_runs = (unsigned int)pl.total_runs; fp.shift = (int)pl.shift;
   fp.step_u = pl.grid / pl.RPU; fp.step_j = pl.grid % pl.RPU;
   fp.step_q = fp.step_u % pl.QT;
