@@ -180,7 +180,9 @@ KVC_API kvc_status kvc_compose(const kvc_desc* desc, const float* scores, int32_
  *   n_keep:  [batch, L] int32,  sum over l == budget exactly, 0 <= n_keep <= N
  *   offsets: [batch, L + 1] int64, exclusive prefix sum of n_keep (offsets[b, L] == budget)
  * composite must be non-increasing in k within a layer (what kvc_compose produces) and
- * non-negative.  0 <= budget <= L * N.
+ * non-negative.  0 <= budget <= L * N.  workspace: kvc_workspace_size bytes (the selection over
+ * pools of more than 128 rows keeps its histograms there; smaller pools are selected by one
+ * kernel on the sorted rows and leave it untouched).
  */
 KVC_API kvc_status kvc_allocate(const kvc_desc* desc, const float* composite, int64_t budget,
                         int32_t* n_keep, int64_t* offsets, void* workspace,
@@ -313,6 +315,15 @@ KVC_API int64_t kvc_launch_count(int32_t reset);
  * that the waits for them run into the bound and the call ends with KVC_ERR_TIMEOUT in its status
  * word (-1: none).  Process-wide; takes effect at the next launch. */
 KVC_API void kvc_debug_score_hooks(int64_t wait_limit_ns, int32_t withhold_unit);
+
+/* Test hook, not for production use: how kvc_allocate (and the allocation inside kvc_compress and
+ * kvc_select_unstructured) finds the threshold of Eqs. 20-22.  path 0: the library chooses (pools of up
+ * to 128 rows: one kernel that narrows windows on the sorted rows; larger pools: the histogram passes of
+ * a radix select); 1: always the histogram passes; 2: the sorted-rows kernel wherever the pool has few
+ * enough rows.  max_rounds bounds the narrowing rounds of that kernel before it falls back to a
+ * bisection over the key range (< 0: the default of 40; 0: bisect at once).  Both ways give identical
+ * results.  Process-wide; takes effect at the next call.  kvc_allocate_static is not affected. */
+KVC_API void kvc_debug_select_hooks(int32_t path, int32_t max_rounds);
 
 /* Library version as major * 10000 + minor * 100 + patch. */
 KVC_API int32_t kvc_version(void);

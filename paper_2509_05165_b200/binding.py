@@ -72,6 +72,8 @@ def _load():
     lib.kvc_score_status_offset.restype = C.c_int
     lib.kvc_debug_score_hooks.argtypes = [i64, i32]
     lib.kvc_debug_score_hooks.restype = None
+    lib.kvc_debug_select_hooks.argtypes = [i32, i32]
+    lib.kvc_debug_select_hooks.restype = None
     lib.kvc_score_uses_tensor_cores.argtypes = [dp]
     lib.kvc_score_uses_tensor_cores.restype = i32
     lib.kvc_score_weighted.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
@@ -187,6 +189,12 @@ def kvc_debug_score_hooks(wait_limit_ns: int = 0, withhold_unit: int = -1) -> No
     """Test hook: bound of the scoring kernel's device-side waits, and a unit whose statistics
     are withheld so that those waits expire.  The defaults restore normal operation."""
     _load().kvc_debug_score_hooks(int(wait_limit_ns), int(withhold_unit))
+
+
+def kvc_debug_select_hooks(path: int = 0, max_rounds: int = -1) -> None:
+    """Test hook: which way the allocation finds its threshold (0 automatic, 1 histogram passes,
+    2 sorted-rows kernel) and the sorted-rows kernel's bound on rounds.  The defaults restore normal operation."""
+    _load().kvc_debug_select_hooks(int(path), int(max_rounds))
 
 
 def kvc_head_sum(desc, scores, head_sum, stream=None) -> None:

@@ -71,5 +71,5 @@ extern "C" kvc_status kvc_allocate_static(const kvc_desc* d, const float* compos
   if ((s = static_scratch(&scratch)) != KVC_OK) return s;
   // launch_allocate zeroes the histograms it uses (stream-ordered) before the first kernel
   return launch_allocate(P, composite, budget, 1, P.min_keep, n_keep, reinterpret_cast<long long*>(offsets), scratch,
-                         kStaticScratchWords * sizeof(unsigned int), (cudaStream_t)stream);
+                         kStaticScratchWords * sizeof(unsigned int), (cudaStream_t)stream, SelectPath::kHistograms);
 }

@@ -133,9 +133,14 @@ size_t allocate_workspace_bytes(const Problem& P);
 // heads_per_row = 1: the pool's rows are the layers, composite [L, Bt, N].  heads_per_row = Hkv (the
 // unstructured variant, App. A.2): the rows are the (layer, head) pairs, composite = the heads'
 // sorted scores [L, Bt, Hkv, N], n_keep [Bt, L * Hkv], offsets [Bt, L * Hkv + 1].
+// How the budget's threshold is found: on the sorted rows by one CTA per sequence (pools of up to 128
+// rows; uses no workspace), or by the histogram passes of a radix select over the workspace.
+enum class SelectPath { kAuto, kHistograms, kSortedRows };
 kvc_status launch_allocate(const Problem& P, const float* composite, long long budget, int heads_per_row,
                            long long min_keep, int32_t* n_keep, long long* offsets, void* ws,
-                           size_t ws_bytes, cudaStream_t st);
+                           size_t ws_bytes, cudaStream_t st, SelectPath path = SelectPath::kAuto);
+// Test hooks: path 0 = automatic, 1 = histograms, 2 = sorted rows where they apply; max_rounds < 0 = default.
+void set_select_hooks(int path, int max_rounds);
 
 // ---- gather -----------------------------------------------------------------------------------
 // Eqs. 23-24.
