@@ -16,12 +16,14 @@
 //                        and count travel in one word, so a reader of the sum needs no fence: the
 //                        word is complete when its count equals the unit's runs.  That is two round
 //                        trips to L2 between the last pass-1 tile of a unit and its first pass-2
-//                        tile.  The long way, for the rows whose word says that some run's sum did
-//                        not fit the fixed-point range (a token about 14 nats above token 0): every
-//                        run also writes its (reference, sum) of every row to global memory before
-//                        it adds to the word, and adds with release semantics; a pass-2 thread that
-//                        needs them acquires the complete word and folds the unit's records of its
-//                        row in run order (the same order for every reader).
+//                        tile.  The long way, for a run's sum that does not fit the fixed-point
+//                        range (a token about 14 nats above token 0): the run writes its
+//                        (reference, sum) of that row to global memory, marks itself in the row's
+//                        bitmap of such runs, and only then counts itself into the word, with
+//                        release semantics (the runs that fit add relaxed and write nothing
+//                        else); a pass-2 thread whose word shows such runs acquires the complete
+//                        word and folds their records, in run order (the same order for every
+//                        reader), into the fixed-point sum of the others.
 //   pass 2 (emit)        the same CTA revisits its tiles a fixed number of runs later, when their
 //                        K rows are still in L2.  D[token, query row] = K Q^T (operands swapped:
 //                        tokens on TMEM lanes), so the max over the window rows (Eq. 14) and the
@@ -86,7 +88,9 @@ struct FastParams {
   CUtensorMap k_maps[kMaxFastLayers];   // K^(l) as (64, N, d / 64, Hkv, Bt), box 64 x 128 x d / 64 x 1 x 1, 128-byte swizzle:
                                         // a tile arrives as d / 64 blocks of 128 rows of 128 bytes with one copy
   CUtensorMap q_maps[kMaxFastLayers];   // Q^(l) as (d, w, Hq, Bt), box 64 x w x G x 1
-  float4* partial;             // [U][RPU][64]: the runs' records: (ref, sum) of rows 2i and 2i+1 of one run
+  float2* partial;             // [U][RPU][128]: (ref, sum) of a row over one run, written only where the sum
+                               // does not fit the row's word
+  unsigned long long* ovf;     // [U][128][4], preset to 0: per row, the runs (bit j) that wrote such a record
   unsigned long long* acc;     // [U][128], preset to 0: per row  arrivals << 56 | overflows << 48 | sum in units
                                // of 2^-20 of 2^(logit - ref[row]), added to by every run of the unit
   const float* ref;            // [U][128]: the row's reference exponent (its scaled logit against token 0)
@@ -273,6 +277,12 @@ __device__ __forceinline__ void named_bar(int id, int threads) {
 // acquires a value of the word that includes this addition)
 __device__ __forceinline__ void red_add_release_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void red_add_relaxed_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void red_or_relaxed_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.or.b64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -662,8 +672,8 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         }
       }
       if (run_ends) {
-        // the two halves of every row meet through shared memory; the lower half's warps write
-        // the run's record of every row and then push its sum
+        // the two halves of every row meet through shared memory; the lower half's warps send the
+        // run's sum of every row
         if (half == 1) *stage = make_float2(row_used ? mref : -INFINITY, row_used ? lsum : 0.f);
         named_bar(3, 256);
         const float2 other = *stage;
@@ -671,17 +681,20 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
         if (half == 0 && ok && c.u != P.withhold_unit) {
           float M = row_used ? mref : -INFINITY, Ls = row_used ? lsum : 0.f;
           combine(M, Ls, other.x, other.y);
-          reinterpret_cast<float2*>(P.partial)[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
-          {
-            // the short way: add the run's sum, rescaled to the row's fixed reference, to the
-            // row's 64-bit word (integer addition: the total does not depend on the order)
-            unsigned long long add = kAccArrival;
-            if (Ls > 0.f) {
-              const float lv = lg2(Ls) + (M - row_ref);                 // log2 of the contribution
-              if (lv < kAccLimitLog2) add += __float2ull_rn(ex2(lv + (float)kAccFracBits));
-              else add += kAccOverflow;                                  // the rows' records decide instead
-            }
-            red_add_release_u64(P.acc + (long long)c.u * kRows + row, add);
+          // the short way: add the run's sum, rescaled to the row's fixed reference, to the row's
+          // 64-bit word (integer addition: the total does not depend on the order)
+          unsigned long long* word = P.acc + (long long)c.u * kRows + row;
+          const float lv = lg2(Ls) + (M - row_ref);                     // log2 of the contribution
+          if (!(Ls > 0.f)) {
+            red_add_relaxed_u64(word, kAccArrival);
+          } else if (lv < kAccLimitLog2) {
+            red_add_relaxed_u64(word, kAccArrival + __float2ull_rn(ex2(lv + (float)kAccFracBits)));
+          } else {
+            // it does not fit: the run's record and its bit in the row's bitmap, then the arrival with
+            // release semantics, so that both are visible to whoever acquires the complete word
+            P.partial[((long long)c.u * P.RPU + c.j) * kRows + row] = make_float2(M, Ls);
+            red_or_relaxed_u64(P.ovf + ((long long)c.u * kRows + row) * 4 + (c.j >> 6), 1ull << (c.j & 63));
+            red_add_release_u64(word, kAccArrival + kAccOverflow);
           }
         }
         mref = -INFINITY; lsum = 0.f;
@@ -739,15 +752,25 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
             }
           }
           if (!pushed) {
-            // the long way: all runs have arrived (the count in the word), and each wrote the row's record
-            // before its release; fold the records in run order (the same order for every reader)
+            // the long way: all runs have arrived (the count in the word); those whose sum did not fit
+            // wrote a record and set their bit before their release.  Fold them, in run order (the same
+            // order for every reader), into the fixed-point sum of the others.
             asm volatile("fence.acq_rel.gpu;" ::: "memory");
-            const float2* rec = reinterpret_cast<const float2*>(P.partial) + (long long)cu.u * P.RPU * kRows + trow;
+            const unsigned long long word = ld_relaxed_u64(P.acc + (long long)cu.u * kRows + trow);
+            const unsigned long long sum = word & kAccSumMask;
             float M = -INFINITY, Ls = 0.f;
-#pragma unroll 4
-            for (int j = 0; j < P.RPU; ++j) {
-              const float2 v = __ldcg(rec + (long long)j * kRows);
-              combine(M, Ls, v.x, v.y);
+            if (sum != 0) { M = early_ref; Ls = (float)sum * 9.5367431640625e-07f; }       // 2^-20
+            const float2* rec = P.partial + (long long)cu.u * P.RPU * kRows + trow;
+            const unsigned long long* bits_of = P.ovf + ((long long)cu.u * kRows + trow) * 4;
+#pragma unroll 1
+            for (int wi = 0; wi < 4; ++wi) {
+              unsigned long long bits = __ldcg(bits_of + wi);
+              while (bits) {
+                const int j = wi * 64 + __ffsll((long long)bits) - 1;
+                bits &= bits - 1;
+                const float2 v = __ldcg(rec + (long long)j * kRows);
+                combine(M, Ls, v.x, v.y);
+              }
             }
             lse = M + log2f(Ls);
           }
@@ -994,6 +1017,7 @@ score_sm100_kernel(const __grid_constant__ FastParams P) {
 struct RefParams {
   int Bt, Hkv, G, HPT, QT, CH, w, d;
   unsigned long long* acc;     // [U][128]: cleared here
+  unsigned long long* ovf;     // [U][128][4]: cleared here
   long long qs0, qs1, qs2, kvs0, kvs1;
   float sl2e;
 };
@@ -1004,6 +1028,11 @@ score_ref_kernel(RefParams P, LayerPtrs qp, LayerPtrs kp, float* __restrict__ re
   const int u = blockIdx.x, row = threadIdx.x;
   // the unit's exchange state: empty words
   P.acc[(long long)u * kRows + row] = 0ull;
+  {
+    ulonglong2* o = reinterpret_cast<ulonglong2*>(P.ovf + ((long long)u * kRows + row) * 4);
+    o[0] = make_ulonglong2(0ull, 0ull);
+    o[1] = make_ulonglong2(0ull, 0ull);
+  }
   const int uh = u / P.QT, qt = u - uh * P.QT;
   const int lb = uh / P.Hkv, h = uh - lb * P.Hkv;
   const int l = lb / P.Bt, b = lb - l * P.Bt;
@@ -1070,7 +1099,7 @@ struct FastPlan {
   int U, NT, RPU, grid, RT;
   int HPT, QT, CH;             // query heads per row tile, row tiles per KV head, row tiles per query head
   long long total_runs, shift;
-  size_t off_partial, off_parts, off_acc, off_ref, off_total;
+  size_t off_partial, off_parts, off_acc, off_ovf, off_ref, off_total;
 };
 
 // sms <= 0: no device yet (host-only size query) -- the workspace does not depend on it
@@ -1098,8 +1127,9 @@ void make_plan(const Problem& P, int sms, FastPlan* pl) {
   const long long lag_runs = (pl->RPU + pl->grid - 1) / pl->grid + 1;
   pl->shift = lag_runs * pl->RT + KVC_SCORE_LAG_TILES;
   size_t off = 0;
-  pl->off_partial = off; off += align_up((size_t)pl->total_runs * 64 * sizeof(float4));
+  pl->off_partial = off; off += align_up((size_t)pl->total_runs * kRows * sizeof(float2));
   pl->off_acc = off; off += align_up((size_t)pl->U * kRows * sizeof(unsigned long long));
+  pl->off_ovf = off; off += align_up((size_t)pl->U * kRows * 4 * sizeof(unsigned long long));
   pl->off_ref = off; off += align_up((size_t)pl->U * kRows * sizeof(float));
   pl->off_parts = off;         // partial group aggregates [QT][L*Bt*Hkv][N], only with several row tiles
   if (pl->QT > 1) off += align_up((size_t)pl->U * P.N * sizeof(float));
@@ -1214,13 +1244,15 @@ kvc_status launch_score_sm100(const Problem& P, const LayerPtrs& q, const LayerP
   }
   char* w = reinterpret_cast<char*>(ws);
 
-  fp.partial = reinterpret_cast<float4*>(w + pl.off_partial);
+  fp.partial = reinterpret_cast<float2*>(w + pl.off_partial);
   fp.acc = reinterpret_cast<unsigned long long*>(w + pl.off_acc);
+  fp.ovf = reinterpret_cast<unsigned long long*>(w + pl.off_ovf);
   float* ref = reinterpret_cast<float*>(w + pl.off_ref);
   fp.ref = ref;
   {
     RefParams rp;
     rp.acc = fp.acc;
+    rp.ovf = fp.ovf;
     rp.Bt = P.Bt; rp.Hkv = P.Hkv; rp.G = G; rp.HPT = pl.HPT; rp.QT = pl.QT; rp.CH = pl.CH; rp.w = P.w; rp.d = P.d;
     rp.qs0 = P.qs[0]; rp.qs1 = P.qs[1]; rp.qs2 = P.qs[2]; rp.kvs0 = P.kvs[0]; rp.kvs1 = P.kvs[1];
     rp.sl2e = P.scale * kLog2eF;
