@@ -423,20 +423,31 @@ merge_runs_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restric
 
 // Eq. 19 over the sorted keys: composite[lb, k] = agg_head_h score(keys[lb, h, k]).
 // Mean: heads added in ascending order in fp32, one division at the end.
+// blockIdx.y = (layer, sequence), blockIdx.x over the ranks.  The heads' keys are fetched eight at a
+// time before they are added, so that a thread waits for memory once, not once per head.
 __global__ void compose_kernel(const uint32_t* __restrict__ keys, float* __restrict__ composite,
-                               int Hkv, long long N, long long total, int agg_head) {
+                               int Hkv, long long N, int agg_head) {
   grid_dependency_wait();
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  const long long lb = i / N, kk = i - lb * N;
+  const long long kk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (kk >= N) return;
+  const long long lb = blockIdx.y;
   const uint32_t* p = keys + lb * Hkv * N + kk;
-  float acc = key_to_score(p[0]);
-  for (int h = 1; h < Hkv; ++h) {
-    const float a = key_to_score(p[(long long)h * N]);
-    acc = (agg_head == KVC_AGG_MAX) ? fmaxf(acc, a) : __fadd_rn(acc, a);
+  float acc = 0.f;
+  for (int h0 = 0; h0 < Hkv; h0 += 8) {
+    uint32_t v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = h0 + j < Hkv ? p[(long long)(h0 + j) * N] : 0u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (h0 + j < Hkv) {
+        const float a = key_to_score(v[j]);
+        if (h0 + j == 0) acc = a;
+        else acc = (agg_head == KVC_AGG_MAX) ? fmaxf(acc, a) : __fadd_rn(acc, a);
+      }
+    }
   }
   if (agg_head == KVC_AGG_MEAN) acc = __fdiv_rn(acc, (float)Hkv);
-  composite[i] = acc;
+  composite[lb * N + kk] = acc;
 }
 
 // Eq. 18 as fp32: the sorted keys turned back into scores.
@@ -555,9 +566,8 @@ kvc_status launch_compose(const Problem& P, const float* scores, int32_t* idx, f
     }
   }
   if (composite == nullptr) return KVC_OK;      // ranking only (the unstructured variant has no Eq. 19)
-  const long long total = (long long)P.L * P.Bt * P.N;
-  KVC_CUDA(launch_dependent(compose_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                            keys_b, composite, P.Hkv, P.N, total, P.agg_head));
+  KVC_CUDA(launch_dependent(compose_kernel, dim3((unsigned)((P.N + 255) / 256), (unsigned)(P.L * P.Bt)), dim3(256), 0, st,
+                            keys_b, composite, P.Hkv, P.N, P.agg_head));
   KVC_LAUNCH_CHECK("compose_kernel");
   return KVC_OK;
 }

@@ -285,6 +285,19 @@ __global__ void score_augment_kernel(float* __restrict__ s, const float* __restr
     }
   }
   if (!augment) return;
+  if (Hkv <= 8) {
+    // all heads' values at once: the thread waits for memory once (added in ascending head order all the same)
+    float v[8];
+#pragma unroll
+    for (int h = 0; h < 8; ++h) v[h] = h < Hkv ? base[(long long)h * N] : 0.f;
+    float sum = 0.f;
+#pragma unroll
+    for (int h = 0; h < 8; ++h) if (h < Hkv) sum += v[h];
+    const float mean = sum / (float)Hkv;
+#pragma unroll
+    for (int h = 0; h < 8; ++h) if (h < Hkv) base[(long long)h * N] = v[h] + mean;
+    return;
+  }
   float sum = 0.f;
   for (int h = 0; h < Hkv; ++h) sum += base[(long long)h * N];
   const float mean = sum / (float)Hkv;
