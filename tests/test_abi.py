@@ -136,3 +136,12 @@ def test_scoring_path_query_and_option_defaults():
     a = kvc.kvc_workspace_size(d3, 10)
     d3.value_norm = 1
     assert kvc.kvc_workspace_size(d3, 10) >= a
+
+
+def test_test_hooks_take_and_restore_their_settings_without_a_device():
+    """The hooks only store process-wide settings; they launch nothing and need no GPU."""
+    kvc.kvc_debug_select_hooks(2, 0)
+    kvc.kvc_debug_select_hooks(1, 5)
+    kvc.kvc_debug_select_hooks()                 # automatic choice, default bound
+    kvc.kvc_debug_score_hooks(1000000, 3)
+    kvc.kvc_debug_score_hooks()                  # default wait bound, nothing withheld
