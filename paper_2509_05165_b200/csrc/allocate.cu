@@ -244,10 +244,11 @@ constexpr int kSelMaxRows = 128;          // rows of a pool this kernel takes (f
 constexpr int kSelDefaultRounds = 40;     // sampling rounds and exact steps together, before the bisection takes over
 
 struct SelectShared {
-  unsigned long long sortbuf[2][kSelThreads];   // exchange buffers of the sort
+  uint32_t sortbuf[2][kSelThreads];             // exchange buffers of the sort
   unsigned long long pref[kSelThreads];         // weighted inclusive ranks, in sorted order
-  long long wt[kSelThreads];                    // block size behind every thread's sample
-  uint32_t skey[kSelThreads];                   // keys in sorted order
+  long long wt[kSelThreads];                    // block size behind every sample
+  uint32_t skey[kSelThreads];                   // the samples' shortened keys in sorted order
+  uint32_t fkey[kSelThreads];                   // the samples' keys
   long long lo[kSelMaxRows], hi[kSelMaxRows];   // the rows' windows: positions < lo are better than T, >= hi worse
   long long gt[kSelMaxRows], ge[kSelMaxRows];   // the answer: entries better than T, and at least as good
   long long off[kSelMaxRows + 1];               // running sum of the window lengths (last step)
@@ -257,18 +258,19 @@ struct SelectShared {
   long long rank, width;                        // T is the rank-th best entry inside the windows (1-based); their total length
   long long slack, new_width;
   unsigned long long tot_lt, tot_le;
-  uint32_t khi;
+  uint32_t khi, khi_key;                        // upper bracket: shortened key, and the key of the sample it came from
+  uint32_t kmin, kmax;                          // range of the round's sample keys
   int ilo;
 };
 
-// Bitonic sort of 1024 values, one per thread; returns the value of rank threadIdx.x (ascending).
+// Bitonic sort of 1024 32-bit values, one per thread; returns the value of rank threadIdx.x (ascending).
 // K0 = 2 for any input; K0 = 2 m when the values arrive as runs of m neighbours that are already
 // sorted, ascending where (threadIdx.x & m) == 0 and descending elsewhere: the stages that would
 // build such runs are left out.  Exchanges closer than a warp go through shuffles, the others
 // through shared memory (two buffers in turn: one barrier per step).  Fully unrolled: every
 // step's partner and direction are constants.
 template <int K0>
-__device__ __forceinline__ unsigned long long block_sort(unsigned long long v, SelectShared& sh) {
+__device__ __forceinline__ uint32_t block_sort(uint32_t v, SelectShared& sh) {
   const int i = threadIdx.x;
   int which = 0;
 #pragma unroll
@@ -276,7 +278,7 @@ __device__ __forceinline__ unsigned long long block_sort(unsigned long long v, S
     const bool asc = (i & k) == 0;
 #pragma unroll
     for (int j = k >> 1; j > 0; j >>= 1) {
-      unsigned long long other;
+      uint32_t other;
       if (j >= 32) {
         sh.sortbuf[which][i] = v;
         __syncthreads();
@@ -362,12 +364,15 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
   // start from runs of S
   const int ks = (tid & S) ? S - 1 - k : k;            // which sample of the row this thread takes
   const unsigned int sample_id = (unsigned int)((r << sshift) | ks);
-  const float* row = composite + row_start(r < R ? r : 0, b, Bt, hpr, N) + floor;
+  const int rr0 = r < R ? r : 0, rl = rr0 / hpr;       // (32-bit: the 64-bit division of row_start is slow)
+  const float* row = composite + (((long long)rl * Bt + b) * hpr + (rr0 - rl * hpr)) * N + floor;
   if (tid < R) { sh.lo[tid] = 0; sh.hi[tid] = M; sh.gt[tid] = 0; sh.ge[tid] = 0; }
   if (tid < kSelMaxRows) { sh.row_a[tid] = 0; sh.row_b[tid] = 0; }
   if (tid == 0) {
     sh.width = (long long)R * M;
     sh.rank = budget < sh.width ? budget : sh.width;
+    sh.kmin = 0xffffffffu;
+    sh.kmax = 0u;
   }
   __syncthreads();
   if (budget > 0 && M > 0) {
@@ -395,13 +400,28 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
         if (k == 0) sh.row_a[r] = w > 0 ? s - 1 : 0;   // what a partial block can hide
       }
       sh.wt[sample_id] = wgt;
-      // (the sample's number inside the row breaks ties, so that equal keys keep the rows' runs sorted)
-      const unsigned long long packed = ((unsigned long long)key << 32) | sample_id;
-      const unsigned long long e = sshift == 5 ? block_sort<64>(packed, sh)
-                                 : sshift == 4 ? block_sort<32>(packed, sh) : block_sort<16>(packed, sh);
-      const uint32_t ekey = (uint32_t)(e >> 32);
+      sh.fkey[sample_id] = key;
+      // The samples are sorted as 32-bit words: the key, taken relative to the smallest sample key and
+      // shortened to its leading 22 bits of the samples' range, above the sample's number (which breaks
+      // ties so that the rows' runs stay sorted).  Shortening is monotone, so every bound below holds
+      // for the shortened keys as it would for the keys; samples that fall together just make the
+      // brackets a little wider.
+      const bool real = wgt > 0;
+      {
+        const uint32_t wmin = __reduce_min_sync(0xffffffffu, real ? key : 0xffffffffu);
+        const uint32_t wmax = __reduce_max_sync(0xffffffffu, real ? key : 0u);
+        if (lane == 0) { atomicMin(&sh.kmin, wmin); atomicMax(&sh.kmax, wmax); }
+      }
+      __syncthreads();
+      const uint32_t base = sh.kmin, span = sh.kmax - base;
+      const int cut = (span >> 22) ? (32 - __clz(span)) - 22 : 0;
+      const uint32_t tkey = real ? ((key - base) >> cut) : 0x3fffffu;
+      const uint32_t packed = (tkey << 10) | sample_id;
+      const uint32_t e = sshift == 5 ? block_sort<64>(packed, sh)
+                       : sshift == 4 ? block_sort<32>(packed, sh) : block_sort<16>(packed, sh);
+      const uint32_t ekey = e >> 10;
       // weighted rank: entries known to be at least as good as this sample (whole blocks only)
-      const unsigned long long P = block_scan((unsigned long long)sh.wt[(int)(e & 0xffffffffu)], sh);
+      const unsigned long long P = block_scan((unsigned long long)sh.wt[e & 1023u], sh);
       sh.skey[tid] = ekey;
       sh.pref[tid] = P;
       if (tid < 32) { const long long v = warp_sum_rows(sh.row_a); if (tid == 0) sh.slack = v; }
@@ -410,7 +430,7 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
       // lower bracket: the last sample value v for which even whole blocks plus one partial block per row
       // hold fewer than `rank` entries at least as good as v: T is worse than v.
       const unsigned long long Pprev = tid ? sh.pref[tid - 1] : 0ull;
-      if (Pprev < (unsigned long long)rank && (unsigned long long)rank <= P) sh.khi = ekey;
+      if (Pprev < (unsigned long long)rank && (unsigned long long)rank <= P) { sh.khi = ekey; sh.khi_key = sh.fkey[e & 1023u]; }
       const long long bound = rank - sh.slack - 1;
       const bool last_of_value = tid == kSelThreads - 1 || sh.skey[tid + 1] != ekey;
       if (last_of_value && (long long)P <= bound) atomicMax(&sh.ilo, tid + 1);
@@ -419,8 +439,8 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
       const int ilo = sh.ilo;
       const uint32_t klo = ilo ? sh.skey[ilo - 1] : 0u;
       // samples of the row on the good side of either bracket (the lanes of a row are neighbours)
-      const uint32_t mlo = __ballot_sync(0xffffffffu, wgt > 0 && ilo > 0 && key <= klo);
-      const uint32_t mhi = __ballot_sync(0xffffffffu, wgt > 0 && key <= khi);
+      const uint32_t mlo = __ballot_sync(0xffffffffu, real && ilo > 0 && tkey <= klo);
+      const uint32_t mhi = __ballot_sync(0xffffffffu, real && tkey <= khi);
       if (r < R && k == 0) {
         long long nlo = lo, nhi = lo;
         if (w > 0) {
@@ -437,20 +457,21 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
       __syncthreads();
       if (tid < 32) {
         const long long taken = warp_sum_rows(sh.row_a), nw = warp_sum_rows(sh.row_b);
-        if (tid == 0) { sh.rank = rank - taken; sh.width = nw; sh.new_width = nw; }
+        if (tid == 0) { sh.rank = rank - taken; sh.width = nw; sh.new_width = nw; sh.kmin = 0xffffffffu; sh.kmax = 0u; }
       }
       __syncthreads();
       const long long new_width = sh.new_width;
       if (new_width > width / 2) {
-        // the windows did not shrink: some value has very many copies.  Locate the upper bracket exactly.
-        locate_in_windows(composite, sh, R, b, Bt, hpr, N, floor, khi);
+        // the windows did not shrink: some value has very many copies (or many keys fell together when
+        // they were shortened).  Locate the key of the upper bracket's sample exactly.
+        locate_in_windows(composite, sh, R, b, Bt, hpr, N, floor, sh.khi_key);
         const long long rk = sh.rank, lt = (long long)sh.tot_lt, le = (long long)sh.tot_le;
         __syncthreads();
         if (rk > lt && rk <= le) { found = true; break; }            // it is T
         if (rk <= lt) {                                               // T is better: the copies leave the windows
           if (tid < R) sh.hi[tid] = sh.gt[tid];
           if (tid == 0) sh.width = lt;
-        } else {                                                      // (cannot happen: T is never worse than the bracket)
+        } else {                                                      // T is worse (only among keys that were shortened alike)
           if (tid < R) sh.lo[tid] = sh.ge[tid];
           if (tid == 0) { sh.rank = rk - le; sh.width = new_width - le; }
         }
@@ -495,9 +516,8 @@ select_sorted_kernel(const float* __restrict__ composite, int R, int Bt, int hpr
           rr = a;
           key = score_to_key(composite[row_start(rr, b, Bt, hpr, N) + floor + sh.lo[rr] + (tid - sh.off[rr])]);
         }
-        const unsigned long long e = block_sort<2>(tid < width ? ((unsigned long long)key << 32) | (unsigned int)tid
-                                                                : ~0ull, sh);
-        if (tid == rank - 1) sh.khi = (uint32_t)(e >> 32);
+        const uint32_t e = block_sort<2>(tid < width ? key : 0xffffffffu, sh);    // (keys alone: T is a value)
+        if (tid == rank - 1) sh.khi = e;
         __syncthreads();
         T = sh.khi;
         if (tid < width) {
